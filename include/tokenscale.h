@@ -1,0 +1,258 @@
+/*
+ * tokenscale.h -- C ABI of the mixed paged-attention step of a Convertible Decoder.
+ *
+ * TokenScale (arXiv 2512.03416) lets a decoder GPU absorb the prefill of burst requests:
+ * every iteration the decoder runs a batch made of its ongoing single-token decode
+ * requests plus (a chunk of) one prefill task, bounded by a profiled "chunk size"
+ * (Sec. 3.4 "Convertible Decoder", Sec. 4.4 "SLO-aware restricted chunked prefill", Eq. 5).
+ * This library is the attention part of that iteration: grouped-query attention over a
+ * paged KV cache (Sec. 2.1: prefill builds the KV cache of all input tokens, decode reuses
+ * it and adds one token per iteration), the append of the step's new K/V into cache pages,
+ * the page bookkeeping, and the per-step token counts that feed Token Velocity (Sec. 3.2, Eq. 1).
+ *
+ * All kernels are CUDA for sm_100a. There is no CPU fallback: a call that has to launch
+ * work returns TS_ERR_CUDA when no usable device is present.
+ *
+ * ---------------------------------------------------------------------------------------
+ * Data layout (frozen; everything is little endian, bf16 = upper 16 bits of an IEEE fp32)
+ *
+ *   KV pool (device, owned by the caller), bf16, index order
+ *        pool[page][kv][head][slot][d]
+ *        page in [0, n_pages), kv in {0 = K, 1 = V}, head in [0, n_kv_heads),
+ *        slot in [0, page_size), d in [0, head_dim)
+ *   element offset = (((page*2 + kv)*n_kv_heads + head)*page_size + slot)*head_dim + d
+ *   One page therefore holds page_size tokens of every KV head, K and V together;
+ *   a (page, kv, head) tile is page_size*head_dim contiguous elements.
+ *
+ *   Token t (0-based position in its request) lives in page block_table[t / page_size],
+ *   slot t % page_size. Slots that hold no token yet are never read or written.
+ *
+ *   Step tensors (device): q and out are [N, n_q_heads, head_dim] bf16, k_new and v_new are
+ *   [N, n_kv_heads, head_dim] bf16, where N = sum of q_len over the rows of the step and the
+ *   rows' tokens are concatenated in row order. Query head h uses KV head h / (n_q_heads / n_kv_heads).
+ *
+ * What a step computes. For row r with ctx = ctx_len[r] cached tokens and q_len[r] new tokens,
+ * new token i (0 <= i < q_len[r]) is appended at position ctx + i and then attends to the
+ * positions 0 .. ctx + i of its own request (all cached context, plus the causal part of the chunk):
+ *        s_j = scale * <q, K_j>,   p_j = exp(s_j - max_j s_j),   out = sum_j p_j V_j / sum_j p_j
+ * with fp32 accumulation and a bf16 (round-to-nearest-even) result.
+ * ---------------------------------------------------------------------------------------
+ */
+#ifndef TOKENSCALE_H_
+#define TOKENSCALE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Return codes. Every entry point returns one of these; nothing throws across the ABI. */
+enum {
+  TS_OK = 0,
+  TS_ERR_INVALID = -1,        /* null pointer, bad handle, bad slot, inconsistent lengths     */
+  TS_ERR_NO_PAGES = -2,       /* the free list cannot cover the request (nothing was taken)   */
+  TS_ERR_NO_SLOT = -3,        /* max_requests requests are already live                       */
+  TS_ERR_TABLE_SHORT = -4,    /* a row's block table does not cover ctx_len + q_len tokens    */
+  TS_ERR_BUDGET = -5,         /* prefill tokens + decode rows of the step exceed chunk_size   */
+  TS_ERR_CUDA = -6,           /* a CUDA runtime call failed (ts_last_cuda_error has the code) */
+  TS_ERR_DEVICE_TIMEOUT = -7, /* a bounded wait inside a kernel ran out                       */
+  TS_ERR_UNSUPPORTED = -8,    /* shape outside what the kernels are built for                 */
+  TS_ERR_WORKSPACE = -9       /* kv_pool or workspace smaller than ts_pool_bytes/ts_workspace_bytes */
+};
+
+typedef struct ts_ctx ts_ctx; /* opaque; host memory; one thread and one stream at a time */
+
+/*
+ * Static description of one decoder instance's attention layer and KV pool.
+ * Supported shapes: head_dim in {64, 128}; page_size == 16; n_q_heads a multiple of
+ * n_kv_heads with a group size n_q_heads / n_kv_heads <= 16.
+ */
+typedef struct {
+  int32_t n_q_heads;          /* Hq                                                            */
+  int32_t n_kv_heads;         /* Hkv                                                           */
+  int32_t head_dim;           /* D                                                             */
+  int32_t page_size;          /* tokens per page; 16                                           */
+  int32_t n_pages;            /* pages in the pool                                             */
+  int32_t max_requests;       /* request slots (rows of the block table)                       */
+  int32_t max_pages_per_req;  /* columns of the block table                                    */
+  int32_t chunk_size;         /* Sec. 4.4: largest allowed (prefill tokens + decode batch size)
+                                 of one step; 0 disables the check                             */
+  int32_t reserved_pages;     /* Eq. 6: pages only ts_alloc_pages(..., for_prefill=1) may take */
+  int32_t decode_split_tokens;/* keys per split of a decode row; 0 = library default; rounded
+                                 up to a multiple of 64                                        */
+  float softmax_scale;        /* 0 => 1/sqrt(head_dim)                                         */
+  int32_t device;             /* CUDA device ordinal that owns kv_pool and workspace           */
+  uint64_t alloc_shuffle_seed;/* 0: free list hands out pages 0,1,2,...; otherwise the initial
+                                 free list is a seeded permutation (scattered pages)           */
+  void* kv_pool;              /* DEVICE, ts_pool_bytes() bytes, caller-owned, 256-byte aligned */
+  size_t kv_pool_bytes;
+  void* workspace;            /* DEVICE scratch, ts_workspace_bytes() bytes, caller-owned,
+                                 256-byte aligned; holds the device block table, the step
+                                 metadata, split partials and the host-buffer staging area     */
+  size_t workspace_bytes;
+} ts_config;
+
+/* Sizes the caller must allocate. Only the shape fields of cfg are read. 0 on a bad shape. */
+size_t ts_pool_bytes(const ts_config* cfg);
+size_t ts_workspace_bytes(const ts_config* cfg);
+
+/*
+ * ts_create: builds the host bookkeeping (free list, block tables, counters). Makes no CUDA
+ * call; kv_pool/workspace may be NULL for host-only use (allocator, planning), in which case
+ * calls that launch return TS_ERR_CUDA. The pool contents are not touched.
+ * ts_destroy: frees host memory and the library's pinned staging buffers; never the pool.
+ */
+int ts_create(const ts_config* cfg, ts_ctx** out);
+int ts_destroy(ts_ctx* ctx);
+
+/*
+ * Requests (Sec. 4.1: the gateway records each request's input length and a predicted
+ * output length). ts_request_add takes a free slot (TS_ERR_NO_SLOT if none) and records the
+ * lengths; no pages are taken yet. expected_output_len is informational (<= 0 if unknown).
+ */
+int ts_request_add(ts_ctx* ctx, int64_t req_id, int32_t prompt_len, int32_t expected_output_len,
+                   int32_t* slot_out);
+
+/*
+ * ts_alloc_pages: grow the slot's block table so that it covers total_tokens tokens
+ * (ceil(total_tokens / page_size) pages). All or nothing: on TS_ERR_NO_PAGES or
+ * TS_ERR_TABLE_SHORT (more than max_pages_per_req) the table is unchanged. for_prefill != 0
+ * may dip into the reserved_pages held back for absorbed prefill work (Eq. 6).
+ * Never shrinks. Host only; the device copy of the table is refreshed by the next step.
+ */
+int ts_alloc_pages(ts_ctx* ctx, int32_t slot, int32_t total_tokens, int32_t for_prefill);
+
+/*
+ * ts_block_table: borrowed, read-only host view of a slot's page list, its page count and the
+ * number of tokens currently cached. Valid until the next call that changes this slot.
+ * Any of the out pointers may be NULL.
+ */
+int ts_block_table(ts_ctx* ctx, int32_t slot, const int32_t** pages_out, int32_t* n_pages_out,
+                   int32_t* n_tokens_out);
+
+/*
+ * ts_block_table_set: replace a slot's page list by the given pages (each in [0, n_pages),
+ * not owned by another slot, no duplicates; pages previously held by the slot return to the
+ * free list first). Lets a caller or a test lay a request out on chosen pages.
+ */
+int ts_block_table_set(ts_ctx* ctx, int32_t slot, const int32_t* pages, int32_t n_pages);
+
+/*
+ * ts_request_free: the request completed. Its pages return to the free list and its length
+ * L_r (tokens cached = prompt + generated) is added to released_tokens: Eq. 1 counts Decode
+ * Velocity as tokens *released* per unit time. The slot becomes reusable.
+ */
+int ts_request_free(ts_ctx* ctx, int32_t slot);
+
+/* ts_request_set_len: overwrite the slot's cached-token count (<= tokens its table covers).
+ * Used to declare context that was written into the pool by other means, or to rewind. */
+int ts_request_set_len(ts_ctx* ctx, int32_t slot, int32_t n_tokens);
+
+/* Step flags */
+enum {
+  TS_STEP_KEEP_LEN = 1 /* do not advance the slots' cached lengths: the same step can be
+                          issued again and rewrites the same bytes (used for timing)         */
+};
+
+/*
+ * One iteration's batch (Sec. 4.4): rows with q_len == 1 are decode requests, rows with
+ * q_len > 1 are prefill chunks. ctx_len[r] must equal the library's cached length of slot[r]
+ * and the slot's table must already cover ctx_len + q_len tokens (ts_alloc_pages), otherwise
+ * the call fails on the host and launches nothing. A slot may appear once per step.
+ * q/k_new/v_new/out: see "Step tensors" above; 16-byte aligned.
+ */
+typedef struct {
+  int32_t n_rows;
+  int32_t flags;
+  const int32_t* slot;    /* HOST [n_rows] */
+  const int32_t* q_len;   /* HOST [n_rows], >= 1 */
+  const int32_t* ctx_len; /* HOST [n_rows], >= 0 */
+  const void* q;          /* DEVICE bf16 [N, Hq, D]  (ts_mixed_step_host: HOST) */
+  const void* k_new;      /* DEVICE bf16 [N, Hkv, D] (ts_mixed_step_host: HOST) */
+  const void* v_new;      /* DEVICE bf16 [N, Hkv, D] (ts_mixed_step_host: HOST) */
+  void* out;              /* DEVICE bf16 [N, Hq, D]  (ts_mixed_step_host: HOST) */
+} ts_step;
+
+/*
+ * ts_kv_append: write the step's new K/V into the rows' pages (Sec. 2.1) and, unless
+ * TS_STEP_KEEP_LEN, advance the cached lengths. q and out are ignored. Asynchronous on
+ * cuda_stream (a cudaStream_t passed as void*; NULL = legacy default stream). Also the way
+ * to load pre-existing context: one row with ctx_len = 0 and q_len = the context length.
+ * Not subject to chunk_size and not counted as a step.
+ */
+int ts_kv_append(ts_ctx* ctx, const ts_step* step, void* cuda_stream);
+
+/*
+ * ts_mixed_step: the decoder iteration. Appends, then runs split-KV decode attention for the
+ * 1-token rows and tiled causal attention for the prefill-chunk rows, merges the splits, and
+ * writes out. Everything is enqueued on cuda_stream; the call does not synchronise.
+ * Enforces Sec. 4.4's budget: (prefill tokens + decode rows) <= chunk_size, else TS_ERR_BUDGET.
+ * Updates the Token Velocity counters. An empty step (n_rows == 0) is TS_OK and launches nothing.
+ */
+int ts_mixed_step(ts_ctx* ctx, const ts_step* step, void* cuda_stream);
+
+/*
+ * ts_mixed_step_host: same step with q, k_new, v_new, out in HOST memory (pinned memory makes
+ * the copies asynchronous). Copies the inputs into the workspace staging area, runs the step,
+ * copies out back and waits for the stream: on return out is valid. N <= chunk_size required
+ * (the staging area is sized by chunk_size; chunk_size must be > 0).
+ */
+int ts_mixed_step_host(ts_ctx* ctx, const ts_step* step, void* cuda_stream);
+
+/*
+ * Token Velocity counters (Sec. 3.2). Cumulative since ts_create; a monitor divides deltas by
+ * its window: prefill velocity = d(prefill_tokens)/dt, generation throughput =
+ * d(decode_tokens)/dt, Decode Velocity (Eq. 1) = d(released_tokens)/dt.
+ * busy_seconds is the sum of caller-reported step times (ts_report_step_time).
+ */
+typedef struct {
+  uint64_t steps;
+  uint64_t prefill_tokens;     /* sum of q_len over rows with q_len > 1                      */
+  uint64_t decode_tokens;      /* number of rows with q_len == 1                             */
+  uint64_t released_tokens;    /* sum of L_r over freed requests (Eq. 1 numerator)           */
+  uint64_t released_requests;
+  uint64_t pages_in_use;
+  uint64_t pages_free;
+  uint64_t kernel_launches;    /* kernels this context has enqueued                          */
+  double busy_seconds;
+} ts_velocity_counters;
+int ts_velocity(ts_ctx* ctx, ts_velocity_counters* out);
+int ts_report_step_time(ts_ctx* ctx, double seconds);
+
+/*
+ * ts_prefill_budget: Eq. 5 per iteration -- the prefill tokens a Convertible Decoder may take
+ * next to decode_batch_size decode rows: max(chunk_size - decode_batch_size, 0).
+ * Dividing by the TPOT SLO gives V_D^{P'}.
+ */
+int32_t ts_prefill_budget(const ts_ctx* ctx, int32_t decode_batch_size);
+
+/*
+ * ts_plan_step: host-only. Validates the step exactly as ts_mixed_step does and writes the
+ * work list it would launch: one record of 8 int32 per work item
+ *   {row, kind (0 decode split, 1 prefill tile), q_begin, q_count, k_begin, k_end,
+ *    partial_slot (-1: writes out directly), reserved}
+ * (token and key positions are relative to the row's request). items may be NULL to query the
+ * count. Returns TS_OK or the validation error; *n_items_out receives the number of items.
+ */
+int ts_plan_step(ts_ctx* ctx, const ts_step* step, int32_t* items, int32_t items_capacity,
+                 int32_t* n_items_out);
+
+/*
+ * ts_last_device_status: waits for cuda_stream, then reads and clears the device status word:
+ * 0, or a bit set of TS_DEV_* flags raised by kernels (they skip the offending access
+ * instead of faulting).
+ */
+enum { TS_DEV_BAD_PAGE = 1, TS_DEV_TIMEOUT = 2 };
+int ts_last_device_status(ts_ctx* ctx, void* cuda_stream, int32_t* status_out);
+
+/* The cudaError_t of the most recent failed CUDA call of this context (0 if none). */
+int ts_last_cuda_error(const ts_ctx* ctx);
+
+const char* ts_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TOKENSCALE_H_ */
