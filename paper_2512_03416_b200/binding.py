@@ -1,0 +1,225 @@
+"""ctypes binding of libtokenscale.so: the same names as include/tokenscale.h, argument
+marshalling only. Every function returns the library's integer code unchanged unless noted.
+
+The library is CUDA-only. If it has not been built, importing symbols from here raises: there
+is no fallback implementation.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+from . import build as _build
+
+TS_OK = 0
+TS_ERR_INVALID = -1
+TS_ERR_NO_PAGES = -2
+TS_ERR_NO_SLOT = -3
+TS_ERR_TABLE_SHORT = -4
+TS_ERR_BUDGET = -5
+TS_ERR_CUDA = -6
+TS_ERR_DEVICE_TIMEOUT = -7
+TS_ERR_UNSUPPORTED = -8
+TS_ERR_WORKSPACE = -9
+TS_STEP_KEEP_LEN = 1
+TS_DEV_BAD_PAGE = 1
+TS_DEV_TIMEOUT = 2
+
+_i32p = ctypes.POINTER(ctypes.c_int32)
+
+
+class ts_config(ctypes.Structure):
+    _fields_ = [("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
+                ("n_pages", ctypes.c_int32), ("max_requests", ctypes.c_int32),
+                ("max_pages_per_req", ctypes.c_int32), ("chunk_size", ctypes.c_int32),
+                ("reserved_pages", ctypes.c_int32), ("decode_split_tokens", ctypes.c_int32),
+                ("softmax_scale", ctypes.c_float), ("device", ctypes.c_int32),
+                ("alloc_shuffle_seed", ctypes.c_uint64),
+                ("kv_pool", ctypes.c_void_p), ("kv_pool_bytes", ctypes.c_size_t),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+
+
+class ts_step(ctypes.Structure):
+    _fields_ = [("n_rows", ctypes.c_int32), ("flags", ctypes.c_int32),
+                ("slot", _i32p), ("q_len", _i32p), ("ctx_len", _i32p),
+                ("q", ctypes.c_void_p), ("k_new", ctypes.c_void_p), ("v_new", ctypes.c_void_p),
+                ("out", ctypes.c_void_p)]
+
+
+class ts_velocity_counters(ctypes.Structure):
+    _fields_ = [("steps", ctypes.c_uint64), ("prefill_tokens", ctypes.c_uint64),
+                ("decode_tokens", ctypes.c_uint64), ("released_tokens", ctypes.c_uint64),
+                ("released_requests", ctypes.c_uint64), ("pages_in_use", ctypes.c_uint64),
+                ("pages_free", ctypes.c_uint64), ("kernel_launches", ctypes.c_uint64),
+                ("busy_seconds", ctypes.c_double)]
+
+
+EXPORTS = ["ts_pool_bytes", "ts_workspace_bytes", "ts_create", "ts_destroy", "ts_request_add",
+           "ts_alloc_pages", "ts_block_table", "ts_block_table_set", "ts_request_free",
+           "ts_request_set_len", "ts_kv_append", "ts_mixed_step", "ts_mixed_step_host",
+           "ts_velocity", "ts_report_step_time", "ts_prefill_budget", "ts_plan_step",
+           "ts_last_device_status", "ts_last_cuda_error", "ts_strerror"]
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB_PATH
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise RuntimeError(
+                f"{path} is missing: build it with `python -m paper_2512_03416_b200.build` "
+                "(needs nvcc); this package has no other implementation")
+        L = ctypes.CDLL(path)
+        cfgp, stepp, vp = ctypes.POINTER(ts_config), ctypes.POINTER(ts_step), ctypes.c_void_p
+        L.ts_pool_bytes.restype = ctypes.c_size_t
+        L.ts_pool_bytes.argtypes = [cfgp]
+        L.ts_workspace_bytes.restype = ctypes.c_size_t
+        L.ts_workspace_bytes.argtypes = [cfgp]
+        L.ts_create.argtypes = [cfgp, ctypes.POINTER(vp)]
+        L.ts_destroy.argtypes = [vp]
+        L.ts_request_add.argtypes = [vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, _i32p]
+        L.ts_alloc_pages.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32]
+        L.ts_block_table.argtypes = [vp, ctypes.c_int32, ctypes.POINTER(_i32p), _i32p, _i32p]
+        L.ts_block_table_set.argtypes = [vp, ctypes.c_int32, _i32p, ctypes.c_int32]
+        L.ts_request_free.argtypes = [vp, ctypes.c_int32]
+        L.ts_request_set_len.argtypes = [vp, ctypes.c_int32, ctypes.c_int32]
+        L.ts_kv_append.argtypes = [vp, stepp, vp]
+        L.ts_mixed_step.argtypes = [vp, stepp, vp]
+        L.ts_mixed_step_host.argtypes = [vp, stepp, vp]
+        L.ts_velocity.argtypes = [vp, ctypes.POINTER(ts_velocity_counters)]
+        L.ts_report_step_time.argtypes = [vp, ctypes.c_double]
+        L.ts_prefill_budget.restype = ctypes.c_int32
+        L.ts_prefill_budget.argtypes = [vp, ctypes.c_int32]
+        L.ts_plan_step.argtypes = [vp, stepp, _i32p, ctypes.c_int32, _i32p]
+        L.ts_last_device_status.argtypes = [vp, vp, _i32p]
+        L.ts_last_cuda_error.argtypes = [vp]
+        L.ts_strerror.restype = ctypes.c_char_p
+        L.ts_strerror.argtypes = [ctypes.c_int]
+        for name in EXPORTS:
+            getattr(L, name)  # AttributeError here means the library is older than the header
+        _lib = L
+    return _lib
+
+
+def ts_pool_bytes(cfg: ts_config) -> int:
+    return lib().ts_pool_bytes(ctypes.byref(cfg))
+
+
+def ts_workspace_bytes(cfg: ts_config) -> int:
+    return lib().ts_workspace_bytes(ctypes.byref(cfg))
+
+
+def ts_create(cfg: ts_config):
+    """Returns (code, handle)."""
+    h = ctypes.c_void_p()
+    rc = lib().ts_create(ctypes.byref(cfg), ctypes.byref(h))
+    return rc, h
+
+
+def ts_destroy(ctx) -> int:
+    return lib().ts_destroy(ctx)
+
+
+def ts_request_add(ctx, req_id: int, prompt_len: int, expected_output_len: int):
+    """Returns (code, slot)."""
+    slot = ctypes.c_int32(-1)
+    rc = lib().ts_request_add(ctx, req_id, prompt_len, expected_output_len, ctypes.byref(slot))
+    return rc, slot.value
+
+
+def ts_alloc_pages(ctx, slot: int, total_tokens: int, for_prefill: int = 0) -> int:
+    return lib().ts_alloc_pages(ctx, slot, total_tokens, for_prefill)
+
+
+def ts_block_table(ctx, slot: int):
+    """Returns (code, pages as a list copy, n_tokens)."""
+    pages = _i32p()
+    n_pages, n_tokens = ctypes.c_int32(0), ctypes.c_int32(0)
+    rc = lib().ts_block_table(ctx, slot, ctypes.byref(pages), ctypes.byref(n_pages), ctypes.byref(n_tokens))
+    if rc != TS_OK:
+        return rc, [], 0
+    return rc, [pages[i] for i in range(n_pages.value)], n_tokens.value
+
+
+def ts_block_table_set(ctx, slot: int, pages) -> int:
+    arr = (ctypes.c_int32 * len(pages))(*[int(p) for p in pages])
+    return lib().ts_block_table_set(ctx, slot, arr, len(pages))
+
+
+def ts_request_free(ctx, slot: int) -> int:
+    return lib().ts_request_free(ctx, slot)
+
+
+def ts_request_set_len(ctx, slot: int, n_tokens: int) -> int:
+    return lib().ts_request_set_len(ctx, slot, n_tokens)
+
+
+def make_step(slots, q_len, ctx_len, q=0, k_new=0, v_new=0, out=0, flags: int = 0):
+    """Marshal host int arrays and raw addresses into a ts_step. Returns (step, keepalive)."""
+    n = len(slots)
+    a_slot = (ctypes.c_int32 * max(n, 1))(*[int(x) for x in slots])
+    a_q = (ctypes.c_int32 * max(n, 1))(*[int(x) for x in q_len])
+    a_c = (ctypes.c_int32 * max(n, 1))(*[int(x) for x in ctx_len])
+    st = ts_step(n, flags, a_slot, a_q, a_c, q or None, k_new or None, v_new or None, out or None)
+    return st, (a_slot, a_q, a_c)
+
+
+def ts_kv_append(ctx, step: ts_step, cuda_stream: int = 0) -> int:
+    return lib().ts_kv_append(ctx, ctypes.byref(step), ctypes.c_void_p(cuda_stream))
+
+
+def ts_mixed_step(ctx, step: ts_step, cuda_stream: int = 0) -> int:
+    return lib().ts_mixed_step(ctx, ctypes.byref(step), ctypes.c_void_p(cuda_stream))
+
+
+def ts_mixed_step_host(ctx, step: ts_step, cuda_stream: int = 0) -> int:
+    return lib().ts_mixed_step_host(ctx, ctypes.byref(step), ctypes.c_void_p(cuda_stream))
+
+
+def ts_velocity(ctx):
+    """Returns (code, dict of counters)."""
+    c = ts_velocity_counters()
+    rc = lib().ts_velocity(ctx, ctypes.byref(c))
+    return rc, {name: getattr(c, name) for name, _ in ts_velocity_counters._fields_}
+
+
+def ts_report_step_time(ctx, seconds: float) -> int:
+    return lib().ts_report_step_time(ctx, seconds)
+
+
+def ts_prefill_budget(ctx, decode_batch_size: int) -> int:
+    return lib().ts_prefill_budget(ctx, decode_batch_size)
+
+
+def ts_plan_step(ctx, step: ts_step):
+    """Returns (code, list of 8-int records)."""
+    n = ctypes.c_int32(0)
+    rc = lib().ts_plan_step(ctx, ctypes.byref(step), None, 0, ctypes.byref(n))
+    if rc != TS_OK or n.value == 0:
+        return rc, []
+    buf = (ctypes.c_int32 * (8 * n.value))()
+    rc = lib().ts_plan_step(ctx, ctypes.byref(step), buf, n.value, ctypes.byref(n))
+    return rc, [tuple(buf[8 * i:8 * i + 8]) for i in range(n.value)]
+
+
+def ts_last_device_status(ctx, cuda_stream: int = 0):
+    """Returns (code, status bits)."""
+    s = ctypes.c_int32(0)
+    rc = lib().ts_last_device_status(ctx, ctypes.c_void_p(cuda_stream), ctypes.byref(s))
+    return rc, s.value
+
+
+def ts_last_cuda_error(ctx) -> int:
+    return lib().ts_last_cuda_error(ctx)
+
+
+def ts_strerror(code: int) -> str:
+    return lib().ts_strerror(code).decode()

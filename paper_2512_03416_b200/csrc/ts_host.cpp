@@ -1,0 +1,689 @@
+// Host side of the mixed paged-attention step: page allocator, per-request block tables,
+// step validation, work-list planning, metadata upload and kernel launches, Token Velocity
+// counters. The public ABI is documented in include/tokenscale.h.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/tokenscale.h"
+#include "ts_internal.h"
+
+namespace {
+
+using ts::CombineItem;
+using ts::TableDelta;
+using ts::WorkItem;
+
+constexpr int kRing = 4;                  // pinned metadata buffers in flight
+constexpr int kDeltaCapacity = 32768;     // table entries per upload batch
+constexpr int kDefaultSplit = 512;        // keys per decode split
+constexpr int kDefaultMaxTokens = 16384;  // step size bound when chunk_size == 0
+constexpr size_t kAlign = 256;
+
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+struct Layout {
+  int max_tokens, max_partials, max_items;
+  size_t off_status, off_table, off_meta, off_delta, off_part_acc, off_part_ml, off_stage;
+  size_t meta_bytes, delta_bytes, stage_q_bytes, stage_kv_bytes, total;
+  // int32 offsets inside the meta area
+  size_t m_row_slot, m_row_ctx, m_row_qlen, m_row_tok0, m_items, m_combines, m_end;
+};
+
+bool shape_ok(const ts_config* c) {
+  if (!c) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->page_size != ts::kPageSize) return false;
+  if (c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->n_q_heads % c->n_kv_heads) return false;
+  if (c->n_q_heads / c->n_kv_heads > ts::kMaxGroup) return false;
+  if (c->n_pages <= 0 || c->max_requests <= 0 || c->max_pages_per_req <= 0) return false;
+  if (c->chunk_size < 0 || c->reserved_pages < 0 || c->decode_split_tokens < 0) return false;
+  return true;
+}
+
+void compute_layout(const ts_config* c, Layout* L) {
+  const int G = c->n_q_heads / c->n_kv_heads;
+  const int R = c->max_requests;
+  L->max_tokens = c->chunk_size > 0 ? c->chunk_size : kDefaultMaxTokens;
+  L->max_partials = 2048 + 2 * R;
+  L->max_items = L->max_partials + R + ceil_div(L->max_tokens * G, ts::kPackedRowsPerTile) + R;
+  size_t m = 0;
+  L->m_row_slot = m; m += R;
+  L->m_row_ctx = m; m += R;
+  L->m_row_qlen = m; m += R;
+  L->m_row_tok0 = m; m += R + 1;
+  m = (m + 7) / 8 * 8;                       // items start 32-byte aligned
+  L->m_items = m; m += (size_t)L->max_items * 8;
+  L->m_combines = m; m += (size_t)R * 4;
+  L->m_end = m;
+  L->meta_bytes = align_up(m * sizeof(int32_t));
+  L->delta_bytes = align_up((size_t)kDeltaCapacity * sizeof(TableDelta));
+  size_t off = 0;
+  L->off_status = off; off += kAlign;
+  L->off_table = off; off += align_up((size_t)R * c->max_pages_per_req * sizeof(int32_t));
+  L->off_meta = off; off += L->meta_bytes;
+  L->off_delta = off; off += L->delta_bytes;
+  L->off_part_acc = off;
+  off += align_up((size_t)L->max_partials * c->n_q_heads * c->head_dim * sizeof(float));
+  L->off_part_ml = off; off += align_up((size_t)L->max_partials * c->n_q_heads * 2 * sizeof(float));
+  L->stage_q_bytes = align_up((size_t)L->max_tokens * c->n_q_heads * c->head_dim * 2);
+  L->stage_kv_bytes = align_up((size_t)L->max_tokens * c->n_kv_heads * c->head_dim * 2);
+  L->off_stage = off; off += 2 * L->stage_q_bytes + 2 * L->stage_kv_bytes;
+  L->total = off;
+}
+
+struct Slot {
+  bool live = false;
+  int64_t req_id = 0;
+  int32_t prompt_len = 0, expected_output_len = 0;
+  int32_t n_pages = 0;       // table entries in use
+  int32_t n_tokens = 0;      // tokens cached
+  int32_t synced_pages = 0;  // leading entries the device copy already holds
+  uint32_t stamp = 0;        // duplicate detection within a step
+};
+
+struct RingBuf {
+  void* host = nullptr;
+  cudaEvent_t ev = nullptr;
+  bool in_flight = false;
+};
+
+uint64_t splitmix64(uint64_t& s) {
+  uint64_t z = (s += 0x9E3779B97F4A7C15ull);
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+}  // namespace
+
+struct ts_ctx {
+  ts_config cfg;
+  Layout L;
+  int G = 1;
+  float scale = 0.f;
+  std::vector<int32_t> table;       // [max_requests][max_pages_per_req]
+  std::vector<Slot> slots;
+  std::vector<int32_t> free_pages;  // stack, next page at the back
+  std::vector<int32_t> page_owner;  // -1 = free
+  std::vector<int32_t> free_slots;  // stack
+  ts_velocity_counters cnt;
+  RingBuf ring[kRing];
+  int ring_next = 0;
+  size_t ring_bytes = 0;
+  bool cuda_ready = false;
+  bool status_cleared = false;
+  int last_cuda_error = 0;
+  uint32_t stamp = 0;
+  // scratch reused across steps
+  std::vector<WorkItem> items;
+  std::vector<CombineItem> combines;
+  std::vector<int32_t> tok0;
+  std::vector<TableDelta> deltas;
+};
+
+namespace {
+
+int32_t* table_row(ts_ctx* c, int slot) { return c->table.data() + (size_t)slot * c->cfg.max_pages_per_req; }
+
+bool slot_ok(const ts_ctx* c, int32_t slot) {
+  return slot >= 0 && slot < c->cfg.max_requests && c->slots[slot].live;
+}
+
+int cuda_fail(ts_ctx* c, cudaError_t e) {
+  c->last_cuda_error = (int)e;
+  return TS_ERR_CUDA;
+}
+
+#define TS_CUDA(c, call)                                 \
+  do {                                                   \
+    cudaError_t e__ = (call);                            \
+    if (e__ != cudaSuccess) return cuda_fail((c), e__);  \
+  } while (0)
+
+void release_pages(ts_ctx* c, int slot) {
+  Slot& s = c->slots[slot];
+  int32_t* row = table_row(c, slot);
+  for (int i = s.n_pages - 1; i >= 0; --i) {
+    c->page_owner[row[i]] = -1;
+    c->free_pages.push_back(row[i]);
+  }
+  s.n_pages = 0;
+  s.synced_pages = 0;
+}
+
+int ensure_cuda(ts_ctx* c, cudaStream_t stream) {
+  if (!c->cfg.kv_pool || !c->cfg.workspace) return cuda_fail(c, cudaErrorInvalidDevicePointer);
+  TS_CUDA(c, cudaSetDevice(c->cfg.device));
+  if (!c->cuda_ready) {
+    c->ring_bytes = std::max(c->L.meta_bytes, c->L.delta_bytes);
+    for (int i = 0; i < kRing; ++i) {
+      TS_CUDA(c, cudaHostAlloc(&c->ring[i].host, c->ring_bytes, cudaHostAllocDefault));
+      TS_CUDA(c, cudaEventCreateWithFlags(&c->ring[i].ev, cudaEventDisableTiming));
+    }
+    c->cuda_ready = true;
+  }
+  if (!c->status_cleared) {
+    TS_CUDA(c, cudaMemsetAsync((char*)c->cfg.workspace + c->L.off_status, 0, kAlign, stream));
+    c->status_cleared = true;
+  }
+  return TS_OK;
+}
+
+// Next pinned buffer; waits only if the copy that last used it has not finished.
+int ring_acquire(ts_ctx* c, RingBuf** out) {
+  RingBuf& r = c->ring[c->ring_next];
+  c->ring_next = (c->ring_next + 1) % kRing;
+  if (r.in_flight) {
+    TS_CUDA(c, cudaEventSynchronize(r.ev));
+    r.in_flight = false;
+  }
+  *out = &r;
+  return TS_OK;
+}
+
+int ring_send(ts_ctx* c, RingBuf* r, size_t dst_off, size_t bytes, cudaStream_t stream) {
+  TS_CUDA(c, cudaMemcpyAsync((char*)c->cfg.workspace + dst_off, r->host, bytes,
+                             cudaMemcpyHostToDevice, stream));
+  TS_CUDA(c, cudaEventRecord(r->ev, stream));
+  r->in_flight = true;
+  return TS_OK;
+}
+
+// Checks shared by ts_kv_append, ts_mixed_step and ts_plan_step. Fills tok0 (prefix sums).
+int validate(ts_ctx* c, const ts_step* st, bool attention, bool need_tensors, int64_t* n_tokens_out,
+             int* n_decode_out, int64_t* n_prefill_out) {
+  if (!c || !st) return TS_ERR_INVALID;
+  if (st->n_rows < 0 || st->n_rows > c->cfg.max_requests) return TS_ERR_INVALID;
+  if (st->n_rows > 0 && (!st->slot || !st->q_len || !st->ctx_len)) return TS_ERR_INVALID;
+  c->tok0.assign((size_t)st->n_rows + 1, 0);
+  ++c->stamp;
+  if (c->stamp == 0) {  // wrapped: restart stamps
+    for (auto& s : c->slots) s.stamp = 0;
+    c->stamp = 1;
+  }
+  int64_t n = 0, n_prefill = 0;
+  int n_decode = 0;
+  const int P = c->cfg.page_size;
+  for (int r = 0; r < st->n_rows; ++r) {
+    const int32_t slot = st->slot[r], ql = st->q_len[r], ctx = st->ctx_len[r];
+    if (!slot_ok(c, slot)) return TS_ERR_INVALID;
+    Slot& s = c->slots[slot];
+    if (s.stamp == c->stamp) return TS_ERR_INVALID;  // slot listed twice
+    s.stamp = c->stamp;
+    if (ql < 1 || ctx < 0) return TS_ERR_INVALID;
+    if (ctx != s.n_tokens) return TS_ERR_INVALID;
+    if ((int64_t)ctx + ql > (int64_t)s.n_pages * P) return TS_ERR_TABLE_SHORT;
+    n += ql;
+    if (n > INT32_MAX / 2) return TS_ERR_INVALID;
+    c->tok0[r + 1] = (int32_t)n;
+    if (ql == 1) ++n_decode; else n_prefill += ql;
+  }
+  if (attention) {
+    if (c->cfg.chunk_size > 0 && n_prefill + n_decode > c->cfg.chunk_size) return TS_ERR_BUDGET;
+    if (n > c->L.max_tokens) return TS_ERR_BUDGET;
+  }
+  if (n > 0 && need_tensors) {
+    if (!st->k_new || !st->v_new) return TS_ERR_INVALID;
+    if (attention && (!st->q || !st->out)) return TS_ERR_INVALID;
+  }
+  *n_tokens_out = n;
+  *n_decode_out = n_decode;
+  *n_prefill_out = n_prefill;
+  return TS_OK;
+}
+
+// Builds c->items / c->combines for a validated step.
+void plan(ts_ctx* c, const ts_step* st) {
+  const int G = c->G;
+  int split = c->cfg.decode_split_tokens > 0 ? c->cfg.decode_split_tokens : kDefaultSplit;
+  split = ceil_div(split, ts::kKeysPerTile) * ts::kKeysPerTile;
+  for (;;) {
+    c->items.clear();
+    c->combines.clear();
+    int partial = 0;
+    for (int r = 0; r < st->n_rows; ++r) {
+      const int ql = st->q_len[r], ctx = st->ctx_len[r];
+      if (ql > 1) {
+        const int rows = ql * G;
+        for (int pr0 = 0; pr0 < rows; pr0 += ts::kPackedRowsPerTile) {
+          const int cnt = std::min(ts::kPackedRowsPerTile, rows - pr0);
+          const int last_tok = (pr0 + cnt - 1) / G;
+          c->items.push_back(WorkItem{r, 1, pr0, cnt, 0, ctx + last_tok + 1, -1, 0});
+        }
+      } else {
+        const int n = ctx + 1;
+        int ns = ceil_div(n, split);
+        if (ns <= 1) {
+          c->items.push_back(WorkItem{r, 0, 0, G, 0, n, -1, 0});
+        } else {
+          const int per = ceil_div(ceil_div(n, ns), ts::kKeysPerTile) * ts::kKeysPerTile;
+          ns = ceil_div(n, per);
+          c->combines.push_back(CombineItem{c->tok0[r], partial, ns, 0});
+          for (int s = 0; s < ns; ++s) {
+            c->items.push_back(WorkItem{r, 0, 0, G, s * per, std::min(n, (s + 1) * per), partial++, 0});
+          }
+        }
+      }
+    }
+    if (partial <= c->L.max_partials) break;
+    split *= 2;
+  }
+  // Heaviest first, so that the tail of the grid is made of short items.
+  auto cost = [](const WorkItem& w) {
+    const int64_t keys = w.k_end - w.k_begin;
+    return w.kind == 1 ? keys * 4 : keys;
+  };
+  std::stable_sort(c->items.begin(), c->items.end(),
+                   [&](const WorkItem& a, const WorkItem& b) { return cost(a) > cost(b); });
+}
+
+// Brings the device copy of the rows' block tables up to date (entries added since the last
+// step that used the slot). Entries travel by value through the pinned ring, so later host-side
+// changes cannot alter what an already enqueued step sees.
+int sync_tables(ts_ctx* c, const ts_step* st, cudaStream_t stream) {
+  c->deltas.clear();
+  for (int r = 0; r < st->n_rows; ++r) {
+    Slot& s = c->slots[st->slot[r]];
+    const int32_t* row = table_row(c, st->slot[r]);
+    for (int i = s.synced_pages; i < s.n_pages; ++i)
+      c->deltas.push_back(TableDelta{st->slot[r], i, row[i]});
+    s.synced_pages = s.n_pages;
+  }
+  size_t at = 0;
+  while (at < c->deltas.size()) {
+    const size_t n = std::min(c->deltas.size() - at, (size_t)kDeltaCapacity);
+    RingBuf* rb;
+    int rc = ring_acquire(c, &rb);
+    if (rc != TS_OK) return rc;
+    std::memcpy(rb->host, c->deltas.data() + at, n * sizeof(TableDelta));
+    rc = ring_send(c, rb, c->L.off_delta, n * sizeof(TableDelta), stream);
+    if (rc != TS_OK) return rc;
+    char* ws = (char*)c->cfg.workspace;
+    TS_CUDA(c, ts::launch_table_update((int32_t*)(ws + c->L.off_table), c->cfg.max_pages_per_req,
+                                       (const TableDelta*)(ws + c->L.off_delta), (int)n, stream));
+    ++c->cnt.kernel_launches;
+    at += n;
+  }
+  return TS_OK;
+}
+
+int upload_meta(ts_ctx* c, const ts_step* st, int n_items, int n_combines, cudaStream_t stream) {
+  RingBuf* rb;
+  int rc = ring_acquire(c, &rb);
+  if (rc != TS_OK) return rc;
+  int32_t* m = (int32_t*)rb->host;
+  const int R = st->n_rows;
+  std::memcpy(m + c->L.m_row_slot, st->slot, sizeof(int32_t) * R);
+  std::memcpy(m + c->L.m_row_ctx, st->ctx_len, sizeof(int32_t) * R);
+  std::memcpy(m + c->L.m_row_qlen, st->q_len, sizeof(int32_t) * R);
+  std::memcpy(m + c->L.m_row_tok0, c->tok0.data(), sizeof(int32_t) * (R + 1));
+  size_t used = c->L.m_row_tok0 + R + 1;
+  if (n_items > 0) {
+    std::memcpy(m + c->L.m_items, c->items.data(), sizeof(WorkItem) * n_items);
+    used = c->L.m_items + (size_t)n_items * 8;
+  }
+  if (n_combines > 0) {
+    std::memcpy(m + c->L.m_combines, c->combines.data(), sizeof(CombineItem) * n_combines);
+    used = c->L.m_combines + (size_t)n_combines * 4;
+  }
+  return ring_send(c, rb, c->L.off_meta, used * sizeof(int32_t), stream);
+}
+
+void fill_device(ts_ctx* c, const ts_step* st, int64_t n_tokens, ts::StepDevice* d) {
+  char* ws = (char*)c->cfg.workspace;
+  const int32_t* meta = (const int32_t*)(ws + c->L.off_meta);
+  d->pool = (uint16_t*)c->cfg.kv_pool;
+  d->table = (int32_t*)(ws + c->L.off_table);
+  d->status = (int32_t*)(ws + c->L.off_status);
+  d->part_acc = (float*)(ws + c->L.off_part_acc);
+  d->part_ml = (float*)(ws + c->L.off_part_ml);
+  d->row_slot = meta + c->L.m_row_slot;
+  d->row_ctx = meta + c->L.m_row_ctx;
+  d->row_qlen = meta + c->L.m_row_qlen;
+  d->row_tok0 = meta + c->L.m_row_tok0;
+  d->items = (const WorkItem*)(meta + c->L.m_items);
+  d->combines = (const CombineItem*)(meta + c->L.m_combines);
+  d->q = (const uint16_t*)st->q;
+  d->k_new = (const uint16_t*)st->k_new;
+  d->v_new = (const uint16_t*)st->v_new;
+  d->out = (uint16_t*)st->out;
+  d->n_rows = st->n_rows;
+  d->n_tokens = (int32_t)n_tokens;
+  d->n_items = 0;
+  d->n_combines = 0;
+  d->Hq = c->cfg.n_q_heads;
+  d->Hkv = c->cfg.n_kv_heads;
+  d->D = c->cfg.head_dim;
+  d->n_pages = c->cfg.n_pages;
+  d->max_pages_per_req = c->cfg.max_pages_per_req;
+  d->scale_log2 = c->scale * 1.4426950408889634f;
+}
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
+  int64_t n_tokens = 0, n_prefill = 0;
+  int n_decode = 0;
+  int rc = validate(c, st, attention, true, &n_tokens, &n_decode, &n_prefill);
+  if (rc != TS_OK) return rc;
+  if (st->n_rows == 0) return TS_OK;
+  if (!aligned16(st->k_new) || !aligned16(st->v_new)) return TS_ERR_INVALID;
+  if (attention && (!aligned16(st->q) || !aligned16(st->out))) return TS_ERR_INVALID;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  if (attention) plan(c, st);
+  rc = ensure_cuda(c, stream);
+  if (rc != TS_OK) return rc;
+  rc = sync_tables(c, st, stream);
+  if (rc != TS_OK) return rc;
+  const int n_items = attention ? (int)c->items.size() : 0;
+  const int n_combines = attention ? (int)c->combines.size() : 0;
+  rc = upload_meta(c, st, n_items, n_combines, stream);
+  if (rc != TS_OK) return rc;
+  ts::StepDevice d;
+  fill_device(c, st, n_tokens, &d);
+  d.n_items = n_items;
+  d.n_combines = n_combines;
+  TS_CUDA(c, ts::launch_kv_append(d, stream));
+  ++c->cnt.kernel_launches;
+  if (attention) {
+    TS_CUDA(c, ts::launch_attention(d, stream));
+    ++c->cnt.kernel_launches;
+    if (n_combines > 0) {
+      TS_CUDA(c, ts::launch_combine(d, stream));
+      ++c->cnt.kernel_launches;
+    }
+    ++c->cnt.steps;
+    c->cnt.prefill_tokens += (uint64_t)n_prefill;
+    c->cnt.decode_tokens += (uint64_t)n_decode;
+  }
+  if (!(st->flags & TS_STEP_KEEP_LEN)) {
+    for (int r = 0; r < st->n_rows; ++r) c->slots[st->slot[r]].n_tokens += st->q_len[r];
+  }
+  return TS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t ts_pool_bytes(const ts_config* cfg) {
+  if (!shape_ok(cfg)) return 0;
+  return (size_t)cfg->n_pages * 2 * cfg->n_kv_heads * cfg->page_size * cfg->head_dim * 2;
+}
+
+size_t ts_workspace_bytes(const ts_config* cfg) {
+  if (!shape_ok(cfg)) return 0;
+  Layout L;
+  compute_layout(cfg, &L);
+  return L.total;
+}
+
+int ts_create(const ts_config* cfg, ts_ctx** out) {
+  if (!out) return TS_ERR_INVALID;
+  *out = nullptr;
+  if (!cfg) return TS_ERR_INVALID;
+  if (!shape_ok(cfg)) return TS_ERR_UNSUPPORTED;
+  if (cfg->reserved_pages > cfg->n_pages) return TS_ERR_INVALID;
+  Layout L;
+  compute_layout(cfg, &L);
+  if (cfg->kv_pool && cfg->kv_pool_bytes < ts_pool_bytes(cfg)) return TS_ERR_WORKSPACE;
+  if (cfg->workspace && cfg->workspace_bytes < L.total) return TS_ERR_WORKSPACE;
+  if (((uintptr_t)cfg->kv_pool | (uintptr_t)cfg->workspace) & (kAlign - 1)) return TS_ERR_INVALID;
+  ts_ctx* c = new (std::nothrow) ts_ctx();
+  if (!c) return TS_ERR_INVALID;
+  c->cfg = *cfg;
+  c->L = L;
+  c->G = cfg->n_q_heads / cfg->n_kv_heads;
+  c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+  c->table.assign((size_t)cfg->max_requests * cfg->max_pages_per_req, -1);
+  c->slots.assign(cfg->max_requests, Slot());
+  c->page_owner.assign(cfg->n_pages, -1);
+  c->free_pages.resize(cfg->n_pages);
+  for (int i = 0; i < cfg->n_pages; ++i) c->free_pages[i] = cfg->n_pages - 1 - i;  // page 0 on top
+  if (cfg->alloc_shuffle_seed) {
+    uint64_t s = cfg->alloc_shuffle_seed;
+    for (int i = cfg->n_pages - 1; i > 0; --i) {
+      const int j = (int)(splitmix64(s) % (uint64_t)(i + 1));
+      std::swap(c->free_pages[i], c->free_pages[j]);
+    }
+  }
+  c->free_slots.resize(cfg->max_requests);
+  for (int i = 0; i < cfg->max_requests; ++i) c->free_slots[i] = cfg->max_requests - 1 - i;
+  std::memset(&c->cnt, 0, sizeof c->cnt);
+  *out = c;
+  return TS_OK;
+}
+
+int ts_destroy(ts_ctx* c) {
+  if (!c) return TS_ERR_INVALID;
+  if (c->cuda_ready) {
+    cudaSetDevice(c->cfg.device);
+    for (int i = 0; i < kRing; ++i) {
+      if (c->ring[i].in_flight) cudaEventSynchronize(c->ring[i].ev);
+      if (c->ring[i].ev) cudaEventDestroy(c->ring[i].ev);
+      if (c->ring[i].host) cudaFreeHost(c->ring[i].host);
+    }
+  }
+  delete c;
+  return TS_OK;
+}
+
+int ts_request_add(ts_ctx* c, int64_t req_id, int32_t prompt_len, int32_t expected_output_len,
+                   int32_t* slot_out) {
+  if (!c || !slot_out || prompt_len < 0) return TS_ERR_INVALID;
+  if (c->free_slots.empty()) return TS_ERR_NO_SLOT;
+  const int slot = c->free_slots.back();
+  c->free_slots.pop_back();
+  Slot& s = c->slots[slot];
+  s = Slot();
+  s.live = true;
+  s.req_id = req_id;
+  s.prompt_len = prompt_len;
+  s.expected_output_len = expected_output_len;
+  *slot_out = slot;
+  return TS_OK;
+}
+
+int ts_alloc_pages(ts_ctx* c, int32_t slot, int32_t total_tokens, int32_t for_prefill) {
+  if (!c || !slot_ok(c, slot) || total_tokens < 0) return TS_ERR_INVALID;
+  Slot& s = c->slots[slot];
+  const int want = ceil_div(total_tokens, c->cfg.page_size);
+  if (want <= s.n_pages) return TS_OK;
+  if (want > c->cfg.max_pages_per_req) return TS_ERR_TABLE_SHORT;
+  const int need = want - s.n_pages;
+  const int64_t usable = (int64_t)c->free_pages.size() - (for_prefill ? 0 : c->cfg.reserved_pages);
+  if (need > usable) return TS_ERR_NO_PAGES;
+  int32_t* row = table_row(c, slot);
+  for (int i = 0; i < need; ++i) {
+    const int32_t p = c->free_pages.back();
+    c->free_pages.pop_back();
+    c->page_owner[p] = slot;
+    row[s.n_pages++] = p;
+  }
+  return TS_OK;
+}
+
+int ts_block_table(ts_ctx* c, int32_t slot, const int32_t** pages_out, int32_t* n_pages_out,
+                   int32_t* n_tokens_out) {
+  if (!c || !slot_ok(c, slot)) return TS_ERR_INVALID;
+  if (pages_out) *pages_out = table_row(c, slot);
+  if (n_pages_out) *n_pages_out = c->slots[slot].n_pages;
+  if (n_tokens_out) *n_tokens_out = c->slots[slot].n_tokens;
+  return TS_OK;
+}
+
+int ts_block_table_set(ts_ctx* c, int32_t slot, const int32_t* pages, int32_t n_pages) {
+  if (!c || !slot_ok(c, slot) || n_pages < 0 || (n_pages > 0 && !pages)) return TS_ERR_INVALID;
+  if (n_pages > c->cfg.max_pages_per_req) return TS_ERR_TABLE_SHORT;
+  // every requested page must be free or already ours, and listed once
+  ++c->stamp;
+  std::vector<char> seen;  // small helper bitmap only for this call
+  seen.assign(c->cfg.n_pages, 0);
+  for (int i = 0; i < n_pages; ++i) {
+    const int32_t p = pages[i];
+    if (p < 0 || p >= c->cfg.n_pages || seen[p]) return TS_ERR_INVALID;
+    if (c->page_owner[p] != -1 && c->page_owner[p] != slot) return TS_ERR_INVALID;
+    seen[p] = 1;
+  }
+  release_pages(c, slot);
+  // remove the requested pages from the free stack, keeping the order of the rest
+  size_t w = 0;
+  for (size_t i = 0; i < c->free_pages.size(); ++i)
+    if (!seen[c->free_pages[i]]) c->free_pages[w++] = c->free_pages[i];
+  c->free_pages.resize(w);
+  Slot& s = c->slots[slot];
+  int32_t* row = table_row(c, slot);
+  for (int i = 0; i < n_pages; ++i) {
+    row[i] = pages[i];
+    c->page_owner[pages[i]] = slot;
+  }
+  s.n_pages = n_pages;
+  s.synced_pages = 0;
+  if (s.n_tokens > n_pages * c->cfg.page_size) s.n_tokens = n_pages * c->cfg.page_size;
+  return TS_OK;
+}
+
+int ts_request_free(ts_ctx* c, int32_t slot) {
+  if (!c || !slot_ok(c, slot)) return TS_ERR_INVALID;
+  Slot& s = c->slots[slot];
+  c->cnt.released_tokens += (uint64_t)s.n_tokens;
+  c->cnt.released_requests += 1;
+  release_pages(c, slot);
+  s.live = false;
+  s.n_tokens = 0;
+  c->free_slots.push_back(slot);
+  return TS_OK;
+}
+
+int ts_request_set_len(ts_ctx* c, int32_t slot, int32_t n_tokens) {
+  if (!c || !slot_ok(c, slot) || n_tokens < 0) return TS_ERR_INVALID;
+  if ((int64_t)n_tokens > (int64_t)c->slots[slot].n_pages * c->cfg.page_size) return TS_ERR_TABLE_SHORT;
+  c->slots[slot].n_tokens = n_tokens;
+  return TS_OK;
+}
+
+int ts_kv_append(ts_ctx* c, const ts_step* st, void* cuda_stream) {
+  return run_step(c, st, cuda_stream, false);
+}
+
+int ts_mixed_step(ts_ctx* c, const ts_step* st, void* cuda_stream) {
+  return run_step(c, st, cuda_stream, true);
+}
+
+int ts_mixed_step_host(ts_ctx* c, const ts_step* st, void* cuda_stream) {
+  if (!c || !st) return TS_ERR_INVALID;
+  if (c->cfg.chunk_size <= 0) return TS_ERR_INVALID;
+  if (st->n_rows == 0) return TS_OK;
+  if (st->n_rows < 0 || !st->q_len) return TS_ERR_INVALID;
+  int64_t n = 0;
+  for (int r = 0; r < st->n_rows; ++r) {
+    if (st->q_len[r] < 1) return TS_ERR_INVALID;
+    n += st->q_len[r];
+    if (n > c->L.max_tokens) return TS_ERR_BUDGET;
+  }
+  if (!st->q || !st->k_new || !st->v_new || !st->out) return TS_ERR_INVALID;
+  if (!c->cfg.workspace) return cuda_fail(c, cudaErrorInvalidDevicePointer);
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  TS_CUDA(c, cudaSetDevice(c->cfg.device));
+  char* ws = (char*)c->cfg.workspace + c->L.off_stage;
+  void* dq = ws;
+  void* dout = ws + c->L.stage_q_bytes;
+  void* dk = ws + 2 * c->L.stage_q_bytes;
+  void* dv = ws + 2 * c->L.stage_q_bytes + c->L.stage_kv_bytes;
+  const size_t qb = (size_t)n * c->cfg.n_q_heads * c->cfg.head_dim * 2;
+  const size_t kb = (size_t)n * c->cfg.n_kv_heads * c->cfg.head_dim * 2;
+  TS_CUDA(c, cudaMemcpyAsync(dq, st->q, qb, cudaMemcpyHostToDevice, stream));
+  TS_CUDA(c, cudaMemcpyAsync(dk, st->k_new, kb, cudaMemcpyHostToDevice, stream));
+  TS_CUDA(c, cudaMemcpyAsync(dv, st->v_new, kb, cudaMemcpyHostToDevice, stream));
+  ts_step dev = *st;
+  dev.q = dq;
+  dev.k_new = dk;
+  dev.v_new = dv;
+  dev.out = dout;
+  const int rc = run_step(c, &dev, cuda_stream, true);
+  if (rc != TS_OK) {
+    cudaStreamSynchronize(stream);  // the input copies may still be reading the caller's buffers
+    return rc;
+  }
+  TS_CUDA(c, cudaMemcpyAsync(st->out, dout, qb, cudaMemcpyDeviceToHost, stream));
+  TS_CUDA(c, cudaStreamSynchronize(stream));
+  return TS_OK;
+}
+
+int ts_velocity(ts_ctx* c, ts_velocity_counters* out) {
+  if (!c || !out) return TS_ERR_INVALID;
+  *out = c->cnt;
+  out->pages_free = c->free_pages.size();
+  out->pages_in_use = (uint64_t)c->cfg.n_pages - c->free_pages.size();
+  return TS_OK;
+}
+
+int ts_report_step_time(ts_ctx* c, double seconds) {
+  if (!c || !(seconds >= 0.0)) return TS_ERR_INVALID;
+  c->cnt.busy_seconds += seconds;
+  return TS_OK;
+}
+
+int32_t ts_prefill_budget(const ts_ctx* c, int32_t decode_batch_size) {
+  if (!c || decode_batch_size < 0) return 0;
+  return std::max(c->cfg.chunk_size - decode_batch_size, 0);
+}
+
+int ts_plan_step(ts_ctx* c, const ts_step* st, int32_t* items, int32_t items_capacity,
+                 int32_t* n_items_out) {
+  if (!n_items_out) return TS_ERR_INVALID;
+  *n_items_out = 0;
+  int64_t n_tokens = 0, n_prefill = 0;
+  int n_decode = 0;
+  // q/out are not needed for planning: validate as an append-only step, then apply the budget.
+  int rc = validate(c, st, false, false, &n_tokens, &n_decode, &n_prefill);
+  if (rc != TS_OK) return rc;
+  if (c->cfg.chunk_size > 0 && n_prefill + n_decode > c->cfg.chunk_size) return TS_ERR_BUDGET;
+  if (n_tokens > c->L.max_tokens) return TS_ERR_BUDGET;
+  plan(c, st);
+  *n_items_out = (int32_t)c->items.size();
+  if (items) {
+    if (items_capacity < (int32_t)c->items.size()) return TS_ERR_INVALID;
+    std::memcpy(items, c->items.data(), c->items.size() * sizeof(WorkItem));
+  }
+  return TS_OK;
+}
+
+int ts_last_device_status(ts_ctx* c, void* cuda_stream, int32_t* status_out) {
+  if (!c || !status_out) return TS_ERR_INVALID;
+  *status_out = 0;
+  if (!c->cfg.workspace) return cuda_fail(c, cudaErrorInvalidDevicePointer);
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  TS_CUDA(c, cudaSetDevice(c->cfg.device));
+  if (!c->status_cleared) return TS_OK;  // nothing has run yet
+  int32_t* dev = (int32_t*)((char*)c->cfg.workspace + c->L.off_status);
+  TS_CUDA(c, cudaMemcpyAsync(status_out, dev, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+  TS_CUDA(c, cudaMemsetAsync(dev, 0, sizeof(int32_t), stream));
+  TS_CUDA(c, cudaStreamSynchronize(stream));
+  return (*status_out & TS_DEV_TIMEOUT) ? TS_ERR_DEVICE_TIMEOUT : TS_OK;
+}
+
+int ts_last_cuda_error(const ts_ctx* c) { return c ? c->last_cuda_error : 0; }
+
+const char* ts_strerror(int code) {
+  switch (code) {
+    case TS_OK: return "ok";
+    case TS_ERR_INVALID: return "invalid argument";
+    case TS_ERR_NO_PAGES: return "not enough free pages";
+    case TS_ERR_NO_SLOT: return "no free request slot";
+    case TS_ERR_TABLE_SHORT: return "block table does not cover the tokens";
+    case TS_ERR_BUDGET: return "step exceeds the chunk size";
+    case TS_ERR_CUDA: return "CUDA runtime error";
+    case TS_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case TS_ERR_UNSUPPORTED: return "unsupported shape";
+    case TS_ERR_WORKSPACE: return "pool or workspace too small";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,74 @@
+// Internal interface between the host scheduler (ts_host.cpp) and the kernels (ts_kernels.cu).
+// Nothing here is part of the public ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ts {
+
+constexpr int kPageSize = 16;
+constexpr int kKeysPerTile = 64;     // keys staged per pipeline stage of the attention kernel
+constexpr int kPackedRowsPerTile = 64;  // (token, head-in-group) rows per prefill work item
+constexpr int kMaxGroup = 16;        // query heads per KV head a decode work item can hold
+
+// One unit of attention work; blockIdx.y supplies the KV head.
+// "Packed rows" enumerate (token, head-in-group) pairs of a request row:
+//   packed row pr -> new token pr / G, query head kv_head*G + pr % G.
+struct WorkItem {
+  int32_t row;          // index into the step's rows
+  int32_t kind;         // 0: decode split, 1: prefill tile
+  int32_t q_begin;      // first packed row
+  int32_t q_count;      // packed rows in this item (decode: G; prefill: <= kPackedRowsPerTile)
+  int32_t k_begin;      // first key position (multiple of kKeysPerTile)
+  int32_t k_end;        // one past the last key position any row of the item may see
+  int32_t partial_slot; // >= 0: write (m, l, acc) partials there; -1: write out directly
+  int32_t reserved;
+};
+static_assert(sizeof(WorkItem) == 32, "WorkItem is 8 int32");
+
+// One entry per token whose splits must be merged.
+struct CombineItem {
+  int32_t token;         // flat token index of the step
+  int32_t first_partial; // first partial slot
+  int32_t n_splits;
+  int32_t reserved;
+};
+
+struct TableDelta {
+  int32_t slot, index, page;
+};
+
+// Device pointers of one step, all inside the caller's workspace unless noted.
+struct StepDevice {
+  // static
+  uint16_t* pool;          // caller's KV pool
+  int32_t* table;          // [max_requests][max_pages_per_req]
+  int32_t* status;         // device status word
+  float* part_acc;         // [max_partials][Hq][D]
+  float* part_ml;          // [max_partials][Hq][2]  (running max in log2 units, sum)
+  // per step (device meta area)
+  const int32_t* row_slot;
+  const int32_t* row_ctx;
+  const int32_t* row_qlen;
+  const int32_t* row_tok0; // [n_rows + 1] prefix sums of q_len
+  const WorkItem* items;
+  const CombineItem* combines;
+  // step tensors
+  const uint16_t* q;
+  const uint16_t* k_new;
+  const uint16_t* v_new;
+  uint16_t* out;
+  // shape
+  int32_t n_rows, n_tokens, n_items, n_combines;
+  int32_t Hq, Hkv, D, n_pages, max_pages_per_req;
+  float scale_log2;        // softmax scale * log2(e)
+};
+
+// Launchers. Each enqueues on `stream` and returns the launch's cudaError_t.
+cudaError_t launch_table_update(int32_t* table, int max_pages_per_req, const TableDelta* deltas,
+                                int n_deltas, cudaStream_t stream);
+cudaError_t launch_kv_append(const StepDevice& s, cudaStream_t stream);
+cudaError_t launch_attention(const StepDevice& s, cudaStream_t stream);
+cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream);
+
+}  // namespace ts
