@@ -222,6 +222,21 @@ int ts_velocity(ts_ctx* ctx, ts_velocity_counters* out);
 int ts_report_step_time(ts_ctx* ctx, double seconds);
 
 /*
+ * Per-kernel device timing, for benchmarks. While enabled, every ts_mixed_step records CUDA
+ * events around its kernels on the step's stream. ts_profile_read waits for the stream, returns
+ * the milliseconds accumulated per kernel over the steps recorded since the last read, and
+ * clears them. Not meant for production steps (each event costs a little stream time).
+ */
+typedef struct {
+  double append_ms;     /* KV append kernel                       */
+  double attention_ms;  /* attention kernel (decode splits + prefill tiles) */
+  double combine_ms;    /* split-combine kernel                   */
+  int64_t steps;
+} ts_profile;
+int ts_profile_enable(ts_ctx* ctx, int enable);
+int ts_profile_read(ts_ctx* ctx, void* cuda_stream, ts_profile* out);
+
+/*
  * ts_prefill_budget: Eq. 5 per iteration -- the prefill tokens a Convertible Decoder may take
  * next to decode_batch_size decode rows: max(chunk_size - decode_batch_size, 0).
  * Dividing by the TPOT SLO gives V_D^{P'}.

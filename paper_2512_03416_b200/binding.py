@@ -55,11 +55,17 @@ class ts_velocity_counters(ctypes.Structure):
                 ("busy_seconds", ctypes.c_double)]
 
 
+class ts_profile(ctypes.Structure):
+    _fields_ = [("append_ms", ctypes.c_double), ("attention_ms", ctypes.c_double),
+                ("combine_ms", ctypes.c_double), ("steps", ctypes.c_int64)]
+
+
 EXPORTS = ["ts_pool_bytes", "ts_workspace_bytes", "ts_create", "ts_destroy", "ts_request_add",
            "ts_alloc_pages", "ts_block_table", "ts_block_table_set", "ts_request_free",
            "ts_request_set_len", "ts_kv_append", "ts_mixed_step", "ts_mixed_step_host",
            "ts_velocity", "ts_report_step_time", "ts_prefill_budget", "ts_plan_step",
-           "ts_last_device_status", "ts_last_cuda_error", "ts_strerror"]
+           "ts_last_device_status", "ts_last_cuda_error", "ts_strerror", "ts_profile_enable",
+           "ts_profile_read"]
 
 _lib = None
 
@@ -101,6 +107,8 @@ def lib() -> ctypes.CDLL:
         L.ts_plan_step.argtypes = [vp, stepp, _i32p, ctypes.c_int32, _i32p]
         L.ts_last_device_status.argtypes = [vp, vp, _i32p]
         L.ts_last_cuda_error.argtypes = [vp]
+        L.ts_profile_enable.argtypes = [vp, ctypes.c_int]
+        L.ts_profile_read.argtypes = [vp, vp, ctypes.POINTER(ts_profile)]
         L.ts_strerror.restype = ctypes.c_char_p
         L.ts_strerror.argtypes = [ctypes.c_int]
         for name in EXPORTS:
@@ -215,6 +223,17 @@ def ts_last_device_status(ctx, cuda_stream: int = 0):
     s = ctypes.c_int32(0)
     rc = lib().ts_last_device_status(ctx, ctypes.c_void_p(cuda_stream), ctypes.byref(s))
     return rc, s.value
+
+
+def ts_profile_enable(ctx, enable: int) -> int:
+    return lib().ts_profile_enable(ctx, enable)
+
+
+def ts_profile_read(ctx, cuda_stream: int = 0):
+    """Returns (code, dict)."""
+    p = ts_profile()
+    rc = lib().ts_profile_read(ctx, ctypes.c_void_p(cuda_stream), ctypes.byref(p))
+    return rc, {name: getattr(p, name) for name, _ in ts_profile._fields_}
 
 
 def ts_last_cuda_error(ctx) -> int:

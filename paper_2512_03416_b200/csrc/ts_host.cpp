@@ -124,6 +124,10 @@ struct ts_ctx {
   std::vector<CombineItem> combines;
   std::vector<int32_t> tok0;
   std::vector<TableDelta> deltas;
+  // optional per-kernel timing: 4 events per recorded step
+  bool profiling = false;
+  std::vector<cudaEvent_t> prof_events;
+  size_t prof_used = 0;
 };
 
 namespace {
@@ -388,15 +392,31 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
   fill_device(c, st, n_tokens, &d);
   d.n_items = n_items;
   d.n_combines = n_combines;
+  cudaEvent_t* pe = nullptr;
+  if (attention && c->profiling) {
+    if (c->prof_used + 4 > c->prof_events.size()) {
+      for (int i = 0; i < 4; ++i) {
+        cudaEvent_t e;
+        TS_CUDA(c, cudaEventCreate(&e));
+        c->prof_events.push_back(e);
+      }
+    }
+    pe = c->prof_events.data() + c->prof_used;
+    c->prof_used += 4;
+    TS_CUDA(c, cudaEventRecord(pe[0], stream));
+  }
   TS_CUDA(c, ts::launch_kv_append(d, stream));
   ++c->cnt.kernel_launches;
   if (attention) {
+    if (pe) TS_CUDA(c, cudaEventRecord(pe[1], stream));
     TS_CUDA(c, ts::launch_attention(d, stream));
     ++c->cnt.kernel_launches;
+    if (pe) TS_CUDA(c, cudaEventRecord(pe[2], stream));
     if (n_combines > 0) {
       TS_CUDA(c, ts::launch_combine(d, stream));
       ++c->cnt.kernel_launches;
     }
+    if (pe) TS_CUDA(c, cudaEventRecord(pe[3], stream));
     ++c->cnt.steps;
     c->cnt.prefill_tokens += (uint64_t)n_prefill;
     c->cnt.decode_tokens += (uint64_t)n_decode;
@@ -469,6 +489,7 @@ int ts_destroy(ts_ctx* c) {
       if (c->ring[i].host) cudaFreeHost(c->ring[i].host);
     }
   }
+  for (cudaEvent_t e : c->prof_events) cudaEventDestroy(e);
   delete c;
   return TS_OK;
 }
@@ -626,6 +647,32 @@ int ts_velocity(ts_ctx* c, ts_velocity_counters* out) {
 int ts_report_step_time(ts_ctx* c, double seconds) {
   if (!c || !(seconds >= 0.0)) return TS_ERR_INVALID;
   c->cnt.busy_seconds += seconds;
+  return TS_OK;
+}
+
+int ts_profile_enable(ts_ctx* c, int enable) {
+  if (!c) return TS_ERR_INVALID;
+  c->profiling = enable != 0;
+  return TS_OK;
+}
+
+int ts_profile_read(ts_ctx* c, void* cuda_stream, ts_profile* out) {
+  if (!c || !out) return TS_ERR_INVALID;
+  std::memset(out, 0, sizeof *out);
+  if (c->prof_used == 0) return TS_OK;
+  TS_CUDA(c, cudaSetDevice(c->cfg.device));
+  TS_CUDA(c, cudaStreamSynchronize((cudaStream_t)cuda_stream));
+  for (size_t i = 0; i + 4 <= c->prof_used; i += 4) {
+    float a = 0.f, b = 0.f, d = 0.f;
+    TS_CUDA(c, cudaEventElapsedTime(&a, c->prof_events[i], c->prof_events[i + 1]));
+    TS_CUDA(c, cudaEventElapsedTime(&b, c->prof_events[i + 1], c->prof_events[i + 2]));
+    TS_CUDA(c, cudaEventElapsedTime(&d, c->prof_events[i + 2], c->prof_events[i + 3]));
+    out->append_ms += a;
+    out->attention_ms += b;
+    out->combine_ms += d;
+    out->steps += 1;
+  }
+  c->prof_used = 0;
   return TS_OK;
 }
 

@@ -127,6 +127,14 @@ class Decoder:
         _check(rc, "ts_velocity")
         return d
 
+    def profile_enable(self, enable: bool) -> None:
+        _check(B.ts_profile_enable(self.ctx, int(enable)), "ts_profile_enable")
+
+    def profile_read(self) -> dict:
+        rc, d = B.ts_profile_read(self.ctx, self._stream())
+        _check(rc, "ts_profile_read")
+        return d
+
     def device_status(self) -> int:
         rc, bits = B.ts_last_device_status(self.ctx, self._stream())
         if rc not in (B.TS_OK, B.TS_ERR_DEVICE_TIMEOUT):

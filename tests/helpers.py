@@ -43,51 +43,23 @@ def parity_metrics(got_f32, want_f32):
 
 
 # ------------------------------------------------------------------------------------ GPU side
-def to_dev(a_u16):
-    """numpy uint16 bit patterns -> int16 CUDA tensor holding the same bits."""
-    import torch
-    return torch.from_numpy(np.ascontiguousarray(a_u16).view(np.int16)).cuda()
-
-
-def from_dev(t):
-    return t.cpu().numpy().view(np.uint16)
-
-
 class GpuRun:
-    """A Decoder loaded with a StepBatch's tables and cached context (through ts_kv_append)."""
+    """LoadedBatch plus the checks every parity test wants after a step."""
 
-    def __init__(self, batch, decode_split_tokens=0, chunk_size=None, max_requests=None, extra_pages=0):
-        import torch
-        from paper_2512_03416_b200.decoder import Decoder
-        s = batch.shape
-        width = max([len(t) for t in batch.tables] + [1]) + extra_pages
-        cs = batch.chunk_size if chunk_size is None else chunk_size
-        self.batch = batch
-        self.dec = Decoder(s.Hq, s.Hkv, s.D, batch.n_pages, max_requests or max(batch.n_rows, 1), width,
-                           chunk_size=cs, decode_split_tokens=decode_split_tokens, nan_fill=True)
-        self.slots = []
-        for r in range(batch.n_rows):
-            slot = self.dec.request_add(1000 + r, int(batch.ctx_len[r]) + int(batch.q_len[r]))
-            self.dec.block_table_set(slot, batch.tables[r])
-            self.slots.append(slot)
-        rows = [r for r in range(batch.n_rows) if batch.ctx_len[r] > 0]
-        if rows:
-            self.dec.kv_append([self.slots[r] for r in rows], [int(batch.ctx_len[r]) for r in rows],
-                               [0] * len(rows), to_dev(batch.context_k), to_dev(batch.context_v))
-        self.q, self.k_new, self.v_new = to_dev(batch.q), to_dev(batch.k_new), to_dev(batch.v_new)
-        self.out = torch.full((batch.n_tokens, s.Hq, s.D), 0x7FC0, dtype=torch.int16, device="cuda")
+    def __init__(self, batch, **kw):
+        from paper_2512_03416_b200.harness import LoadedBatch
+        self.lb = LoadedBatch(batch, **kw)
+        self.dec = self.lb.dec
+        self.slots = self.lb.slots
 
     def step(self, keep_len=False):
-        import torch
-        b = self.batch
-        self.dec.mixed_step(self.slots, b.q_len.tolist(), b.ctx_len.tolist(), self.q, self.k_new, self.v_new,
-                            self.out, keep_len=keep_len)
-        torch.cuda.synchronize()
+        self.lb.step(keep_len=keep_len)
+        out = self.lb.output()
         assert self.dec.device_status() == 0
-        return wl.bf16_bits_to_f32(from_dev(self.out))
+        return out
 
     def pool(self):
-        return from_dev(self.dec.pool)
+        return self.lb.pool()
 
 
 def assert_parity(got, want, profile="paper", what=""):
