@@ -262,6 +262,49 @@ int ts_plan_step(ts_ctx* ctx, const ts_step* step, int32_t* items, int32_t items
 enum { TS_DEV_BAD_PAGE = 1, TS_DEV_TIMEOUT = 2 };
 int ts_last_device_status(ts_ctx* ctx, void* cuda_stream, int32_t* status_out);
 
+/*
+ * ts_decode_attention_static: decode attention (one query token per row) that allocates
+ * nothing and needs no workspace. (The paper has no counterpart; this is a packaging variant
+ * of the split-KV decode path of ts_mixed_step.)
+ *
+ * Who it is for: code that must not, or cannot, obtain device memory at the point where it
+ * needs attention -- for example a serving process whose framework has already claimed all
+ * of HBM for its own KV pool, so that a further cudaMalloc would fail; a plug-in that is only
+ * handed tensors and is not allowed to own memory; or a latency-critical loop that cannot
+ * afford the device-wide synchronisation an allocation may imply. Such a caller cannot supply
+ * the workspace ts_create asks for. Here the split partials and the work list live in a
+ * fixed array inside the library (about 8.6 MiB, present on every GPU that loads the
+ * library, until the process ends). The call makes no cudaMalloc/cudaFree and uses no
+ * allocating routine.
+ *
+ * Arguments (all tensors DEVICE memory of `device`, owned by the caller):
+ *   kv_pool       the pool in the layout documented above; the K/V of every attended token,
+ *                 the newest one included, must already be in it (this call appends nothing)
+ *   block_tables  int32 [n_rows][table_width]: page ids of row r in its first
+ *                 ceil(kv_len[r]/16) entries
+ *   kv_len        int32 [n_rows]: tokens row r attends to, 1 <= kv_len[r] <= 16*table_width
+ *                 (a row outside this range is not processed and its output is NaN)
+ *   q, out        bf16 [n_rows, n_q_heads, head_dim], 16-byte aligned
+ *   n_splits      keys of each row are cut into at most this many splits (1..16)
+ *   softmax_scale 0 => 1/sqrt(head_dim)
+ * Limits of the built-in scratch: n_rows <= 256, n_splits <= 16 and
+ * n_rows * n_splits * n_q_heads * head_dim <= 2^21; beyond them the call returns
+ * TS_ERR_WORKSPACE and launches nothing. Shapes as for ts_config, else TS_ERR_UNSUPPORTED.
+ *
+ * The work is enqueued on cuda_stream and the call returns without waiting. The first call on
+ * a device looks up the device address of the built-in array (it makes `device` current, as
+ * every call does); make that first call outside any stream capture.
+ * All calls in the process share the one array and it keeps the previous call's contents
+ * (each call rewrites every entry it later reads, so nothing needs clearing by the caller):
+ * two calls whose kernels can overlap on the GPU -- different streams, or different host
+ * threads -- race on it. Keep calls on one stream, or order them with events.
+ */
+int ts_decode_attention_static(int32_t device, int32_t n_q_heads, int32_t n_kv_heads,
+                               int32_t head_dim, int32_t n_pages, const void* kv_pool,
+                               const int32_t* block_tables, int32_t table_width,
+                               const int32_t* kv_len, int32_t n_rows, int32_t n_splits,
+                               float softmax_scale, const void* q, void* out, void* cuda_stream);
+
 /* The cudaError_t of the most recent failed CUDA call of this context (0 if none). */
 int ts_last_cuda_error(const ts_ctx* ctx);
 

@@ -65,7 +65,7 @@ EXPORTS = ["ts_pool_bytes", "ts_workspace_bytes", "ts_create", "ts_destroy", "ts
            "ts_request_set_len", "ts_kv_append", "ts_mixed_step", "ts_mixed_step_host",
            "ts_velocity", "ts_report_step_time", "ts_prefill_budget", "ts_plan_step",
            "ts_last_device_status", "ts_last_cuda_error", "ts_strerror", "ts_profile_enable",
-           "ts_profile_read"]
+           "ts_profile_read", "ts_decode_attention_static"]
 
 _lib = None
 
@@ -109,6 +109,9 @@ def lib() -> ctypes.CDLL:
         L.ts_last_cuda_error.argtypes = [vp]
         L.ts_profile_enable.argtypes = [vp, ctypes.c_int]
         L.ts_profile_read.argtypes = [vp, vp, ctypes.POINTER(ts_profile)]
+        L.ts_decode_attention_static.argtypes = [
+            ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp,
+            ctypes.c_int32, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_float, vp, vp, vp]
         L.ts_strerror.restype = ctypes.c_char_p
         L.ts_strerror.argtypes = [ctypes.c_int]
         for name in EXPORTS:
@@ -234,6 +237,18 @@ def ts_profile_read(ctx, cuda_stream: int = 0):
     p = ts_profile()
     rc = lib().ts_profile_read(ctx, ctypes.c_void_p(cuda_stream), ctypes.byref(p))
     return rc, {name: getattr(p, name) for name, _ in ts_profile._fields_}
+
+
+def ts_decode_attention_static(device: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n_pages: int,
+                               kv_pool: int, block_tables: int, table_width: int, kv_len: int,
+                               n_rows: int, n_splits: int, softmax_scale: float, q: int, out: int,
+                               cuda_stream: int = 0) -> int:
+    """Decode attention that uses the library's built-in scratch; pointers are raw device addresses."""
+    return lib().ts_decode_attention_static(device, n_q_heads, n_kv_heads, head_dim, n_pages,
+                                            ctypes.c_void_p(kv_pool), ctypes.c_void_p(block_tables),
+                                            table_width, ctypes.c_void_p(kv_len), n_rows, n_splits,
+                                            softmax_scale, ctypes.c_void_p(q), ctypes.c_void_p(out),
+                                            ctypes.c_void_p(cuda_stream))
 
 
 def ts_last_cuda_error(ctx) -> int:

@@ -420,3 +420,150 @@ cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream) {
 }
 
 }  // namespace ts
+
+// ------------------------------------------------------------------------------------------
+// ts_decode_attention_static: split-KV decode attention whose scratch (split partials and the
+// work list) sits in a fixed device array of this library instead of caller-provided memory.
+// It reuses the attention and combine kernels above unchanged; only the planning is different
+// (done on the device, a fixed number of splits per row).
+// ------------------------------------------------------------------------------------------
+namespace ts {
+namespace {
+
+constexpr int kStaticMaxRows = 256;
+constexpr int kStaticMaxSplits = 16;
+constexpr size_t kStaticAccFloats = size_t(1) << 21;               // 8 MiB of split accumulators
+constexpr size_t kStaticMlFloats = kStaticAccFloats / 64 * 2;      // (max, sum) per (slot, head), D >= 64
+constexpr size_t kStaticItems = size_t(kStaticMaxRows) * kStaticMaxSplits;
+
+struct StaticScratch {
+  float part_acc[kStaticAccFloats];
+  float part_ml[kStaticMlFloats];
+  WorkItem items[kStaticItems];
+  CombineItem combines[kStaticMaxRows];
+  int32_t row_slot[kStaticMaxRows];
+  int32_t row_ctx[kStaticMaxRows];
+  int32_t row_tok0[kStaticMaxRows + 1];
+  int32_t status;
+};
+
+// Lives in every context that loads the library, until the process exits (about 8.6 MiB).
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+// One thread per (row, split): writes the row arrays, the work items and the combine list.
+__global__ void static_plan_kernel(StaticScratch* sc, const int32_t* kv_len, int n_rows, int n_splits,
+                                   int G, int table_width) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx == 0) sc->status = 0;
+  if (idx >= n_rows * n_splits) return;
+  const int r = idx / n_splits, s = idx % n_splits;
+  const int n = kv_len[r];
+  const bool ok = n >= 1 && n <= table_width * kPageSize;
+  int per = 0, ns = 0;
+  if (ok) {
+    per = ((n + n_splits - 1) / n_splits + kKeysPerTile - 1) / kKeysPerTile * kKeysPerTile;
+    ns = (n + per - 1) / per;
+  }
+  WorkItem it;
+  it.row = r;
+  it.kind = 0;
+  it.q_begin = 0;
+  it.reserved = 0;
+  if (s < ns) {
+    it.q_count = G;
+    it.k_begin = s * per;
+    it.k_end = min(n, (s + 1) * per);
+    it.partial_slot = r * n_splits + s;
+  } else {          // nothing to do: zero query rows and an empty key range
+    it.q_count = 0;
+    it.k_begin = 0;
+    it.k_end = 0;
+    it.partial_slot = -1;
+  }
+  sc->items[idx] = it;
+  if (s == 0) {
+    sc->row_slot[r] = r;
+    sc->row_ctx[r] = ok ? n - 1 : 0;
+    sc->row_tok0[r] = r;
+    if (r == n_rows - 1) sc->row_tok0[n_rows] = n_rows;
+    CombineItem c;
+    c.token = r;
+    c.first_partial = r * n_splits;
+    c.n_splits = ns;       // 0 for a rejected row: its output becomes NaN
+    c.reserved = 0;
+    sc->combines[r] = c;
+  }
+}
+
+constexpr int kMaxDevices = 64;
+StaticScratch* g_static_ptr[kMaxDevices] = {};
+
+}  // namespace
+}  // namespace ts
+
+extern "C" int ts_decode_attention_static(int32_t device, int32_t n_q_heads, int32_t n_kv_heads,
+                                          int32_t head_dim, int32_t n_pages, const void* kv_pool,
+                                          const int32_t* block_tables, int32_t table_width,
+                                          const int32_t* kv_len, int32_t n_rows, int32_t n_splits,
+                                          float softmax_scale, const void* q, void* out,
+                                          void* cuda_stream) {
+  using namespace ts;
+  if (n_rows == 0) return TS_OK;
+  if (!kv_pool || !block_tables || !kv_len || !q || !out) return TS_ERR_INVALID;
+  if (device < 0 || device >= kMaxDevices || n_rows < 0 || n_pages <= 0 || table_width <= 0)
+    return TS_ERR_INVALID;
+  if (head_dim != 64 && head_dim != 128) return TS_ERR_UNSUPPORTED;
+  if (n_q_heads <= 0 || n_kv_heads <= 0 || n_q_heads % n_kv_heads) return TS_ERR_UNSUPPORTED;
+  const int G = n_q_heads / n_kv_heads;
+  if (G > kMaxGroup) return TS_ERR_UNSUPPORTED;
+  if (((uintptr_t)q | (uintptr_t)out | (uintptr_t)kv_pool) & 15u) return TS_ERR_INVALID;
+  // the built-in scratch is fixed: refuse what does not fit
+  if (n_rows > kStaticMaxRows || n_splits < 1 || n_splits > kStaticMaxSplits) return TS_ERR_WORKSPACE;
+  if ((size_t)n_rows * n_splits * n_q_heads * head_dim > kStaticAccFloats) return TS_ERR_WORKSPACE;
+
+  if (cudaSetDevice(device) != cudaSuccess) return TS_ERR_CUDA;
+  if (!g_static_ptr[device]) {
+    // In host code the array's name is not a device address; ask the runtime for the address
+    // of this device's copy, once, with the device current.
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return TS_ERR_CUDA;
+    g_static_ptr[device] = static_cast<StaticScratch*>(p);
+  }
+  StaticScratch* sc = g_static_ptr[device];
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+  const int n_items = n_rows * n_splits;
+  static_plan_kernel<<<(n_items + 127) / 128, 128, 0, stream>>>(sc, kv_len, n_rows, n_splits, G, table_width);
+  if (cudaGetLastError() != cudaSuccess) return TS_ERR_CUDA;
+
+  StepDevice d;
+  d.pool = (uint16_t*)kv_pool;            // only read by these kernels
+  d.table = (int32_t*)block_tables;       // only read
+  d.status = &sc->status;
+  d.part_acc = sc->part_acc;
+  d.part_ml = sc->part_ml;
+  d.row_slot = sc->row_slot;
+  d.row_ctx = sc->row_ctx;
+  d.row_qlen = nullptr;                   // not read by attention / combine
+  d.row_tok0 = sc->row_tok0;
+  d.items = sc->items;
+  d.combines = sc->combines;
+  d.q = (const uint16_t*)q;
+  d.k_new = nullptr;
+  d.v_new = nullptr;
+  d.out = (uint16_t*)out;
+  d.n_rows = n_rows;
+  d.n_tokens = n_rows;
+  d.n_items = n_items;
+  d.n_combines = n_rows;
+  d.Hq = n_q_heads;
+  d.Hkv = n_kv_heads;
+  d.D = head_dim;
+  d.n_pages = n_pages;
+  d.max_pages_per_req = table_width;
+  const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+  d.scale_log2 = scale * 1.4426950408889634f;
+  if (launch_attention(d, stream) != cudaSuccess) return TS_ERR_CUDA;
+  if (launch_combine(d, stream) != cudaSuccess) return TS_ERR_CUDA;
+  return TS_OK;
+}
