@@ -116,6 +116,9 @@ struct ts_ctx {
   int ring_next = 0;
   size_t ring_bytes = 0;
   bool cuda_ready = false;
+  CUtensorMap kv_map;               // TMA view of the pool for the decode kernel
+  int n_sms = 0;
+  int n_prefill_items = 0;          // of the current plan
   bool status_cleared = false;
   int last_cuda_error = 0;
   uint32_t stamp = 0;
@@ -160,6 +163,30 @@ void release_pages(ts_ctx* c, int slot) {
   s.synced_pages = 0;
 }
 
+// 5-D tensor map over the pool, fastest dimension first: head_dim, slot, KV head, K|V, page.
+// One box = 64 elements (128 bytes, the swizzle span) x 16 slots x 1 head x {K, V} x 1 page.
+int make_kv_map(ts_ctx* c) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                               CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                               CUtensorMapFloatOOBfill);
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  TS_CUDA(c, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (!fn || qres != cudaDriverEntryPointSuccess) return cuda_fail(c, cudaErrorNotSupported);
+  const cuuint64_t D = c->cfg.head_dim, P = c->cfg.page_size, H = c->cfg.n_kv_heads;
+  const cuuint64_t dims[5] = {D, P, H, 2, (cuuint64_t)c->cfg.n_pages};
+  const cuuint64_t strides[4] = {D * 2, P * D * 2, H * P * D * 2, 2 * H * P * D * 2};
+  const cuuint32_t box[5] = {64, (cuuint32_t)P, 1, 2, 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  const CUresult r = ((EncodeFn)fn)(&c->kv_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, c->cfg.kv_pool, dims,
+                                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return cuda_fail(c, cudaErrorInvalidValue);
+  return TS_OK;
+}
+
 int ensure_cuda(ts_ctx* c, cudaStream_t stream) {
   if (!c->cfg.kv_pool || !c->cfg.workspace) return cuda_fail(c, cudaErrorInvalidDevicePointer);
   TS_CUDA(c, cudaSetDevice(c->cfg.device));
@@ -169,6 +196,9 @@ int ensure_cuda(ts_ctx* c, cudaStream_t stream) {
       TS_CUDA(c, cudaHostAlloc(&c->ring[i].host, c->ring_bytes, cudaHostAllocDefault));
       TS_CUDA(c, cudaEventCreateWithFlags(&c->ring[i].ev, cudaEventDisableTiming));
     }
+    TS_CUDA(c, cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->cfg.device));
+    int rc = make_kv_map(c);
+    if (rc != TS_OK) return rc;
     c->cuda_ready = true;
   }
   if (!c->status_cleared) {
@@ -277,13 +307,14 @@ void plan(ts_ctx* c, const ts_step* st) {
     if (partial <= c->L.max_partials) break;
     split *= 2;
   }
-  // Heaviest first, so that the tail of the grid is made of short items.
-  auto cost = [](const WorkItem& w) {
-    const int64_t keys = w.k_end - w.k_begin;
-    return w.kind == 1 ? keys * 4 : keys;
-  };
-  std::stable_sort(c->items.begin(), c->items.end(),
-                   [&](const WorkItem& a, const WorkItem& b) { return cost(a) > cost(b); });
+  // Prefill tiles first, then decode splits; inside each group heaviest first, so that the tail
+  // of each launch is made of short items.
+  std::stable_sort(c->items.begin(), c->items.end(), [](const WorkItem& a, const WorkItem& b) {
+    if (a.kind != b.kind) return a.kind > b.kind;
+    return (a.k_end - a.k_begin) > (b.k_end - b.k_begin);
+  });
+  c->n_prefill_items = 0;
+  for (const WorkItem& w : c->items) c->n_prefill_items += w.kind == 1;
 }
 
 // Brings the device copy of the rows' block tables up to date (entries added since the last
@@ -360,6 +391,7 @@ void fill_device(ts_ctx* c, const ts_step* st, int64_t n_tokens, ts::StepDevice*
   d->n_tokens = (int32_t)n_tokens;
   d->n_items = 0;
   d->n_combines = 0;
+  d->n_prefill_items = 0;
   d->Hq = c->cfg.n_q_heads;
   d->Hkv = c->cfg.n_kv_heads;
   d->D = c->cfg.head_dim;
@@ -409,8 +441,17 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
   ++c->cnt.kernel_launches;
   if (attention) {
     if (pe) TS_CUDA(c, cudaEventRecord(pe[1], stream));
-    TS_CUDA(c, ts::launch_attention(d, stream));
-    ++c->cnt.kernel_launches;
+    d.n_prefill_items = c->n_prefill_items;
+    if (c->n_prefill_items > 0) {
+      ts::StepDevice dp = d;
+      dp.n_items = c->n_prefill_items;
+      TS_CUDA(c, ts::launch_attention(dp, stream));
+      ++c->cnt.kernel_launches;
+    }
+    if (n_items > c->n_prefill_items) {
+      TS_CUDA(c, ts::launch_decode(d, c->kv_map, c->n_sms, stream));
+      ++c->cnt.kernel_launches;
+    }
     if (pe) TS_CUDA(c, cudaEventRecord(pe[2], stream));
     if (n_combines > 0) {
       TS_CUDA(c, ts::launch_combine(d, stream));

@@ -1,6 +1,7 @@
 // Internal interface between the host scheduler (ts_host.cpp) and the kernels (ts_kernels.cu).
 // Nothing here is part of the public ABI.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -60,6 +61,7 @@ struct StepDevice {
   uint16_t* out;
   // shape
   int32_t n_rows, n_tokens, n_items, n_combines;
+  int32_t n_prefill_items;  // items[0, n_prefill_items) are prefill tiles, the rest decode splits
   int32_t Hq, Hkv, D, n_pages, max_pages_per_req;
   float scale_log2;        // softmax scale * log2(e)
 };
@@ -70,5 +72,8 @@ cudaError_t launch_table_update(int32_t* table, int max_pages_per_req, const Tab
 cudaError_t launch_kv_append(const StepDevice& s, cudaStream_t stream);
 cudaError_t launch_attention(const StepDevice& s, cudaStream_t stream);
 cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream);
+// Decode splits items[n_prefill_items, n_items): persistent kernel, one CTA per SM, K/V pages by TMA
+// through kv_map (5-D view of the pool: head_dim, slot, KV head, K|V, page; box 64 x 16 x 1 x 2 x 1).
+cudaError_t launch_decode(const StepDevice& s, const CUtensorMap& kv_map, int n_sms, cudaStream_t stream);
 
 }  // namespace ts

@@ -556,6 +556,7 @@ extern "C" int ts_decode_attention_static(int32_t device, int32_t n_q_heads, int
   d.n_tokens = n_rows;
   d.n_items = n_items;
   d.n_combines = n_rows;
+  d.n_prefill_items = 0;
   d.Hq = n_q_heads;
   d.Hkv = n_kv_heads;
   d.D = head_dim;
