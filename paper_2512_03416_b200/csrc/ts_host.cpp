@@ -50,7 +50,7 @@ void compute_layout(const ts_config* c, Layout* L) {
   const int R = c->max_requests;
   L->max_tokens = c->chunk_size > 0 ? c->chunk_size : kDefaultMaxTokens;
   L->max_partials = 2048 + 2 * R;
-  L->max_items = L->max_partials + R + ceil_div(L->max_tokens * G, ts::kPackedRowsPerTile) + R;
+  L->max_items = L->max_partials + R + ceil_div(L->max_tokens, std::max(1, ts::kPackedRowsPerTile / G)) + R;
   size_t m = 0;
   L->m_row_slot = m; m += R;
   L->m_row_ctx = m; m += R;
@@ -116,7 +116,9 @@ struct ts_ctx {
   int ring_next = 0;
   size_t ring_bytes = 0;
   bool cuda_ready = false;
-  CUtensorMap kv_map;               // TMA view of the pool for the decode kernel
+  CUtensorMap kv_map;               // TMA view of the pool, box = K and V of one (page, head) half
+  CUtensorMap kv1_map;              // same view, box = K or V only (prefill operand tiles)
+  void* encode_fn = nullptr;        // cuTensorMapEncodeTiled
   int n_sms = 0;
   int n_prefill_items = 0;          // of the current plan
   bool status_cleared = false;
@@ -163,26 +165,44 @@ void release_pages(ts_ctx* c, int slot) {
   s.synced_pages = 0;
 }
 
-// 5-D tensor map over the pool, fastest dimension first: head_dim, slot, KV head, K|V, page.
-// One box = 64 elements (128 bytes, the swizzle span) x 16 slots x 1 head x {K, V} x 1 page.
-int make_kv_map(ts_ctx* c) {
-  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                               CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                               CUtensorMapFloatOOBfill);
-  void* fn = nullptr;
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 5-D tensor maps over the pool, fastest dimension first: head_dim, slot, KV head, K|V, page.
+// Box = 64 elements (128 bytes, the swizzle span) x 16 slots x 1 head x {K and V | one of them} x 1 page.
+int make_kv_maps(ts_ctx* c) {
   cudaDriverEntryPointQueryResult qres;
-  TS_CUDA(c, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
-  if (!fn || qres != cudaDriverEntryPointSuccess) return cuda_fail(c, cudaErrorNotSupported);
+  TS_CUDA(c, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_fn, cudaEnableDefault, &qres));
+  if (!c->encode_fn || qres != cudaDriverEntryPointSuccess) return cuda_fail(c, cudaErrorNotSupported);
   const cuuint64_t D = c->cfg.head_dim, P = c->cfg.page_size, H = c->cfg.n_kv_heads;
   const cuuint64_t dims[5] = {D, P, H, 2, (cuuint64_t)c->cfg.n_pages};
   const cuuint64_t strides[4] = {D * 2, P * D * 2, H * P * D * 2, 2 * H * P * D * 2};
-  const cuuint32_t box[5] = {64, (cuuint32_t)P, 1, 2, 1};
   const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-  const CUresult r = ((EncodeFn)fn)(&c->kv_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, c->cfg.kv_pool, dims,
-                                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  for (int both = 0; both < 2; ++both) {
+    const cuuint32_t box[5] = {64, (cuuint32_t)P, 1, both ? 2u : 1u, 1};
+    const CUresult r = ((EncodeFn)c->encode_fn)(both ? &c->kv_map : &c->kv1_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                                                5, c->cfg.kv_pool, dims, strides, box, estr,
+                                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail(c, cudaErrorInvalidValue);
+  }
+  return TS_OK;
+}
+
+// q viewed as (head_dim, head in group, KV head, token); one box = 64 elements x G heads x 1 x
+// 128/G tokens = one 64-column half of a 128-row query tile in packed (token, head) order.
+int make_q_map(ts_ctx* c, const void* q, int64_t n_tokens, CUtensorMap* out) {
+  const cuuint64_t D = c->cfg.head_dim, G = c->G, H = c->cfg.n_kv_heads;
+  const cuuint64_t dims[4] = {D, G, H, (cuuint64_t)n_tokens};
+  const cuuint64_t strides[3] = {D * 2, G * D * 2, H * G * D * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)G, 1, (cuuint32_t)(ts::kPackedRowsTc / c->G)};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult r = ((EncodeFn)c->encode_fn)(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q), dims,
+                                              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return cuda_fail(c, cudaErrorInvalidValue);
   return TS_OK;
 }
@@ -197,7 +217,7 @@ int ensure_cuda(ts_ctx* c, cudaStream_t stream) {
       TS_CUDA(c, cudaEventCreateWithFlags(&c->ring[i].ev, cudaEventDisableTiming));
     }
     TS_CUDA(c, cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->cfg.device));
-    int rc = make_kv_map(c);
+    int rc = make_kv_maps(c);
     if (rc != TS_OK) return rc;
     c->cuda_ready = true;
   }
@@ -283,23 +303,24 @@ void plan(ts_ctx* c, const ts_step* st) {
     for (int r = 0; r < st->n_rows; ++r) {
       const int ql = st->q_len[r], ctx = st->ctx_len[r];
       if (ql > 1) {
-        const int rows = ql * G;
-        for (int pr0 = 0; pr0 < rows; pr0 += ts::kPackedRowsPerTile) {
-          const int cnt = std::min(ts::kPackedRowsPerTile, rows - pr0);
-          const int last_tok = (pr0 + cnt - 1) / G;
-          c->items.push_back(WorkItem{r, 1, pr0, cnt, 0, ctx + last_tok + 1, -1, 0});
+        // tile = as many whole tokens as fit the kernel's packed rows (128 for head_dim 128, else 64)
+        const int tile_rows = c->cfg.head_dim == 128 ? ts::kPackedRowsTc : ts::kPackedRowsPerTile;
+        const int tt = tile_rows / G;
+        for (int t0 = 0; t0 < ql; t0 += tt) {
+          const int cnt = std::min(tt, ql - t0);
+          c->items.push_back(WorkItem{r, 1, t0, cnt, 0, ctx + t0 + cnt, -1, 0});
         }
       } else {
         const int n = ctx + 1;
         int ns = ceil_div(n, split);
         if (ns <= 1) {
-          c->items.push_back(WorkItem{r, 0, 0, G, 0, n, -1, 0});
+          c->items.push_back(WorkItem{r, 0, 0, 1, 0, n, -1, 0});
         } else {
           const int per = ceil_div(ceil_div(n, ns), ts::kKeysPerTile) * ts::kKeysPerTile;
           ns = ceil_div(n, per);
           c->combines.push_back(CombineItem{c->tok0[r], partial, ns, 0});
           for (int s = 0; s < ns; ++s) {
-            c->items.push_back(WorkItem{r, 0, 0, G, s * per, std::min(n, (s + 1) * per), partial++, 0});
+            c->items.push_back(WorkItem{r, 0, 0, 1, s * per, std::min(n, (s + 1) * per), partial++, 0});
           }
         }
       }
@@ -443,9 +464,16 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
     if (pe) TS_CUDA(c, cudaEventRecord(pe[1], stream));
     d.n_prefill_items = c->n_prefill_items;
     if (c->n_prefill_items > 0) {
-      ts::StepDevice dp = d;
-      dp.n_items = c->n_prefill_items;
-      TS_CUDA(c, ts::launch_attention(dp, stream));
+      if (c->cfg.head_dim == 128) {
+        CUtensorMap q_map;
+        rc = make_q_map(c, st->q, n_tokens, &q_map);
+        if (rc != TS_OK) return rc;
+        TS_CUDA(c, ts::launch_prefill(d, c->kv1_map, q_map, stream));
+      } else {
+        ts::StepDevice dp = d;
+        dp.n_items = c->n_prefill_items;
+        TS_CUDA(c, ts::launch_attention(dp, stream));
+      }
       ++c->cnt.kernel_launches;
     }
     if (n_items > c->n_prefill_items) {

@@ -9,17 +9,18 @@ namespace ts {
 
 constexpr int kPageSize = 16;
 constexpr int kKeysPerTile = 64;     // keys staged per pipeline stage of the attention kernel
-constexpr int kPackedRowsPerTile = 64;  // (token, head-in-group) rows per prefill work item
+constexpr int kPackedRowsPerTile = 64;  // (token, head) rows of a prefill tile, head_dim 64 path
+constexpr int kPackedRowsTc = 128;      // (token, head) rows of a prefill tile, tcgen05 path (head_dim 128)
 constexpr int kMaxGroup = 16;        // query heads per KV head a decode work item can hold
 
-// One unit of attention work; blockIdx.y supplies the KV head.
-// "Packed rows" enumerate (token, head-in-group) pairs of a request row:
-//   packed row pr -> new token pr / G, query head kv_head*G + pr % G.
+// One unit of attention work; the KV head comes from the grid.
+// Inside a kernel the (token, head-in-group) pairs of an item are "packed rows":
+//   packed row pr -> token q_begin + pr / G, query head kv_head*G + pr % G.
 struct WorkItem {
   int32_t row;          // index into the step's rows
   int32_t kind;         // 0: decode split, 1: prefill tile
-  int32_t q_begin;      // first packed row
-  int32_t q_count;      // packed rows in this item (decode: G; prefill: <= kPackedRowsPerTile)
+  int32_t q_begin;      // first new token of the row this item covers (decode: 0)
+  int32_t q_count;      // tokens in this item (decode: 1; prefill: tile_rows / G at most)
   int32_t k_begin;      // first key position (multiple of kKeysPerTile)
   int32_t k_end;        // one past the last key position any row of the item may see
   int32_t partial_slot; // >= 0: write (m, l, acc) partials there; -1: write out directly
@@ -74,6 +75,10 @@ cudaError_t launch_attention(const StepDevice& s, cudaStream_t stream);
 cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream);
 // Decode splits items[n_prefill_items, n_items): persistent kernel, one CTA per SM, K/V pages by TMA
 // through kv_map (5-D view of the pool: head_dim, slot, KV head, K|V, page; box 64 x 16 x 1 x 2 x 1).
+// Prefill tiles items[0, n_prefill_items), head_dim 128: tcgen05/TMEM kernel. kv1_map is the pool view
+// with box 64 x 16 x 1 x 1 x 1; q_map views q as (head_dim, G, KV head, token), box 64 x G x 1 x 128/G.
+cudaError_t launch_prefill(const StepDevice& s, const CUtensorMap& kv1_map, const CUtensorMap& q_map,
+                           cudaStream_t stream);
 cudaError_t launch_decode(const StepDevice& s, const CUtensorMap& kv_map, int n_sms, cudaStream_t stream);
 
 }  // namespace ts

@@ -246,8 +246,9 @@ __global__ void __launch_bounds__(kThreads, 2) attention_kernel(StepDevice s) {
   // The 16 packed rows of this warp: decode -> all warps share rows 0..15; prefill -> 16 each.
   const int row_base = decode ? 0 : warp * 16;
   const int r0 = row_base + (lane >> 2), r1 = r0 + 8;
-  const bool real0 = r0 < it.q_count, real1 = r1 < it.q_count;
-  const int pr0 = it.q_begin + r0, pr1 = it.q_begin + r1;
+  const int n_packed = it.q_count * G;                  // packed rows of this item
+  const bool real0 = r0 < n_packed, real1 = r1 < n_packed;
+  const int pr0 = it.q_begin * G + r0, pr1 = it.q_begin * G + r1;
   const int tokA = pr0 / G, headA = kv_head * G + pr0 % G;
   const int tokB = pr1 / G, headB = kv_head * G + pr1 % G;
   const int lim0 = real0 ? min(ctx + tokA + 1, it.k_end) : it.k_end;
@@ -351,7 +352,7 @@ __global__ void __launch_bounds__(kThreads, 2) attention_kernel(StepDevice s) {
     }
   }
   __syncthreads();
-  for (int idx = tid; idx < it.q_count * D; idx += kThreads) {
+  for (int idx = tid; idx < n_packed * D; idx += kThreads) {
     const int r = idx / D, d = idx % D;
     float mm = sm_m[r];
 #pragma unroll
@@ -363,7 +364,7 @@ __global__ void __launch_bounds__(kThreads, 2) attention_kernel(StepDevice s) {
       ll += wgt * sm_l[w * 16 + r];
       acc += wgt * sm_o[(w * 16 + r) * D + d];
     }
-    const int pr = it.q_begin + r;
+    const int pr = it.q_begin * G + r;
     const int head = kv_head * G + pr % G;
     const int tok = tok0 + pr / G;
     if (it.partial_slot < 0) {
@@ -470,7 +471,7 @@ __global__ void static_plan_kernel(StaticScratch* sc, const int32_t* kv_len, int
   it.q_begin = 0;
   it.reserved = 0;
   if (s < ns) {
-    it.q_count = G;
+    it.q_count = 1;
     it.k_begin = s * per;
     it.k_end = min(n, (s + 1) * per);
     it.partial_slot = r * n_splits + s;

@@ -77,3 +77,23 @@ def test_split_count_invariance(split):
     want, _ = oracle_step(b)
     got = GpuRun(b, decode_split_tokens=split).step()
     assert_parity(got, want, "peaked", f"split {split}")
+
+
+@pytest.mark.parametrize("profile", ["paper", "peaked", "needle"])
+def test_config3_burst_8b(profile):
+    b = wl.config3(profile=profile)
+    want, pool_want = oracle_step(b)
+    run = GpuRun(b)
+    got = run.step()
+    assert_parity(got, want, profile, f"config3/{profile}")
+    assert np.array_equal(run.pool(), pool_want)
+
+
+@pytest.mark.parametrize("profile", ["paper", "needle"])
+def test_config4_chunked_8b(profile):
+    b = wl.config4(profile=profile)
+    want, pool_want = oracle_step(b)
+    run = GpuRun(b)
+    got = run.step()
+    assert_parity(got, want, profile, f"config4/{profile}")
+    assert np.array_equal(run.pool(), pool_want)

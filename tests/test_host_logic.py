@@ -163,7 +163,7 @@ def test_step_validation_launches_nothing():
     B.ts_destroy(h)
 
 
-def _check_plan(items, G, rows):
+def _check_plan(items, G, rows, tile_rows=128):
     """Every (packed query row, key) pair of the step is covered exactly once."""
     by_row = {}
     for it in items:
@@ -172,7 +172,7 @@ def _check_plan(items, G, rows):
     for r, (ql, ctx) in enumerate(rows):
         its = by_row.pop(r)
         if ql == 1:
-            assert all(i[1] == 0 and i[2] == 0 and i[3] == G for i in its)
+            assert all(i[1] == 0 and i[2] == 0 and i[3] == 1 for i in its)
             spans = sorted((i[4], i[5]) for i in its)
             assert spans[0][0] == 0 and spans[-1][1] == ctx + 1
             assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
@@ -188,10 +188,10 @@ def _check_plan(items, G, rows):
             tiles = sorted((i[2], i[3], i[5]) for i in its)
             at = 0
             for q0, cnt, k_end in tiles:
-                assert q0 == at and 1 <= cnt <= 64
+                assert q0 == at and 1 <= cnt <= tile_rows // G
                 at += cnt
-                assert k_end == ctx + (q0 + cnt - 1) // G + 1
-            assert at == ql * G
+                assert k_end == ctx + q0 + cnt
+            assert at == ql
     assert not by_row
     assert len(set(partials)) == len(partials)
 
@@ -228,7 +228,7 @@ def test_planner_respects_partial_capacity():
     rc, items = B.ts_plan_step(h, B.make_step(slots, [1] * 256, ctxs)[0])
     assert rc == B.TS_OK
     assert max(i[6] for i in items) < 2048 + 2 * 256       # split grew until the partials fit
-    _check_plan(items, 1, [(1, 16000)] * 256)
+    _check_plan(items, 1, [(1, 16000)] * 256, 64)
     B.ts_destroy(h)
 
 
