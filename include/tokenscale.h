@@ -249,7 +249,7 @@ int32_t ts_prefill_budget(const ts_ctx* ctx, int32_t decode_batch_size);
  *   {row, kind (0 decode split, 1 prefill tile), q_begin, q_count, k_begin, k_end,
  *    partial_slot (-1: writes out directly), reserved}
  * q_begin/q_count: the new tokens of the row the item covers (a decode split: 0, 1; a prefill
- * tile: 128/G tokens at most for head_dim 128, 64/G for head_dim 64); the item attends keys
+ * tile: 2*(128/G) tokens at most for head_dim 128, 64/G for head_dim 64); the item attends keys
  * [k_begin, k_end), each token only up to its own position.
  * (token and key positions are relative to the row's request). items may be NULL to query the
  * count. Returns TS_OK or the validation error; *n_items_out receives the number of items.

@@ -117,7 +117,6 @@ struct ts_ctx {
   size_t ring_bytes = 0;
   bool cuda_ready = false;
   CUtensorMap kv_map;               // TMA view of the pool, box = K and V of one (page, head) half
-  CUtensorMap kv1_map;              // same view, box = K or V only (prefill operand tiles)
   void* encode_fn = nullptr;        // cuTensorMapEncodeTiled
   int n_sms = 0;
   int n_prefill_items = 0;          // of the current plan
@@ -169,8 +168,8 @@ typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void
                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// 5-D tensor maps over the pool, fastest dimension first: head_dim, slot, KV head, K|V, page.
-// Box = 64 elements (128 bytes, the swizzle span) x 16 slots x 1 head x {K and V | one of them} x 1 page.
+// 5-D tensor map over the pool, fastest dimension first: head_dim, slot, KV head, K|V, page.
+// Box = 64 elements (128 bytes, the swizzle span) x 16 slots x 1 head x {K, V} x 1 page.
 int make_kv_maps(ts_ctx* c) {
   cudaDriverEntryPointQueryResult qres;
   TS_CUDA(c, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_fn, cudaEnableDefault, &qres));
@@ -179,15 +178,12 @@ int make_kv_maps(ts_ctx* c) {
   const cuuint64_t dims[5] = {D, P, H, 2, (cuuint64_t)c->cfg.n_pages};
   const cuuint64_t strides[4] = {D * 2, P * D * 2, H * P * D * 2, 2 * H * P * D * 2};
   const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-  for (int both = 0; both < 2; ++both) {
-    const cuuint32_t box[5] = {64, (cuuint32_t)P, 1, both ? 2u : 1u, 1};
-    const CUresult r = ((EncodeFn)c->encode_fn)(both ? &c->kv_map : &c->kv1_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
-                                                5, c->cfg.kv_pool, dims, strides, box, estr,
-                                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return cuda_fail(c, cudaErrorInvalidValue);
-  }
+  const cuuint32_t box[5] = {64, (cuuint32_t)P, 1, 2, 1};
+  const CUresult r = ((EncodeFn)c->encode_fn)(&c->kv_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, c->cfg.kv_pool,
+                                              dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return cuda_fail(c, cudaErrorInvalidValue);
   return TS_OK;
 }
 
@@ -303,9 +299,9 @@ void plan(ts_ctx* c, const ts_step* st) {
     for (int r = 0; r < st->n_rows; ++r) {
       const int ql = st->q_len[r], ctx = st->ctx_len[r];
       if (ql > 1) {
-        // tile = as many whole tokens as fit the kernel's packed rows (128 for head_dim 128, else 64)
-        const int tile_rows = c->cfg.head_dim == 128 ? ts::kPackedRowsTc : ts::kPackedRowsPerTile;
-        const int tt = tile_rows / G;
+        // head_dim 128: two query tiles of 128 packed rows per item (128/G whole tokens each);
+        // head_dim 64: one tile of 64 packed rows
+        const int tt = c->cfg.head_dim == 128 ? 2 * (ts::kPackedRowsTc / G) : ts::kPackedRowsPerTile / G;
         for (int t0 = 0; t0 < ql; t0 += tt) {
           const int cnt = std::min(tt, ql - t0);
           c->items.push_back(WorkItem{r, 1, t0, cnt, 0, ctx + t0 + cnt, -1, 0});
@@ -468,7 +464,7 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
         CUtensorMap q_map;
         rc = make_q_map(c, st->q, n_tokens, &q_map);
         if (rc != TS_OK) return rc;
-        TS_CUDA(c, ts::launch_prefill(d, c->kv1_map, q_map, stream));
+        TS_CUDA(c, ts::launch_prefill(d, q_map, stream));
       } else {
         ts::StepDevice dp = d;
         dp.n_items = c->n_prefill_items;

@@ -75,10 +75,9 @@ cudaError_t launch_attention(const StepDevice& s, cudaStream_t stream);
 cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream);
 // Decode splits items[n_prefill_items, n_items): persistent kernel, one CTA per SM, K/V pages by TMA
 // through kv_map (5-D view of the pool: head_dim, slot, KV head, K|V, page; box 64 x 16 x 1 x 2 x 1).
-// Prefill tiles items[0, n_prefill_items), head_dim 128: tcgen05/TMEM kernel. kv1_map is the pool view
-// with box 64 x 16 x 1 x 1 x 1; q_map views q as (head_dim, G, KV head, token), box 64 x G x 1 x 128/G.
-cudaError_t launch_prefill(const StepDevice& s, const CUtensorMap& kv1_map, const CUtensorMap& q_map,
-                           cudaStream_t stream);
+// Prefill tiles items[0, n_prefill_items), head_dim 128: tcgen05/TMEM kernel.
+// q_map views q as (head_dim, G, KV head, token), box 64 x G x 1 x 128/G.
+cudaError_t launch_prefill(const StepDevice& s, const CUtensorMap& q_map, cudaStream_t stream);
 cudaError_t launch_decode(const StepDevice& s, const CUtensorMap& kv_map, int n_sms, cudaStream_t stream);
 
 }  // namespace ts

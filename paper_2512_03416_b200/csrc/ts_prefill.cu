@@ -1,15 +1,19 @@
 // Causal prefill-chunk attention on the 5th-generation tensor cores (sm_100a, head_dim 128).
 //
-// One CTA = one tile of 128 packed query rows (128/G consecutive tokens x the G query heads of
-// one KV head) against all keys the tile may see, 128 keys per block:
+// One CTA = one work item = two query tiles A and B of 128 packed rows each (128/G consecutive
+// tokens x the G query heads of one KV head per tile) against all keys they may see, 128 keys per
+// block. Per tile and block:
 //     S = Q K^T   (tcgen05.mma, operands in 128B-swizzled shared memory, fp32 accumulator in TMEM)
 //     online softmax by one warpgroup, one query row per thread, straight out of TMEM
 //     O += P V    (tcgen05.mma, P read from TMEM as bf16, V from shared memory, O accumulates in TMEM)
-// Warp roles: warps 0-3 softmax / epilogue (thread i owns TMEM lane i), warp 4 TMA producer,
-// warp 5 MMA issuer and TMEM owner. K and V blocks come page by page (16 keys) through TMA with
-// the page id as a coordinate; S is double buffered so that Q K^T of block j+1 overlaps the
-// softmax of block j. The O rescale is lazy: the reference maximum of a row only moves when the
-// new maximum exceeds it by more than 2^8, so most blocks never touch O.
+// The two tiles share every K/V block (half the shared-memory fill per flop) and run out of phase:
+// while one tile's warpgroup is in its softmax, the tensor pipe works for the other tile.
+// TMEM (512 columns): S_A, S_B, O_A, O_B, 128 columns each; P overwrites the first 64 columns of
+// its S. Warp roles: warps 0-3 softmax/epilogue of tile A, warps 4-7 of tile B (thread = TMEM lane =
+// query row), warps 8-9 K loaders, warps 10-11 V loaders (16-byte cp.async through the block table
+// into the swizzled operand layout), warp 12 MMA issuer and TMEM owner; the Q tiles come by TMA.
+// The O rescale is lazy: a row's reference maximum only moves when the new maximum exceeds it by
+// more than 2^8, so most blocks never touch O.
 // Every mbarrier wait is bounded; a wait that runs out raises TS_DEV_TIMEOUT and the CTA drains.
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -21,33 +25,35 @@
 namespace ts {
 namespace {
 
-constexpr int kPfThreads = 192;
+constexpr int kPfThreads = 416;                 // 8 softmax warps + 4 loader warps + MMA warp
+constexpr int kLoaderThreads = 64;              // per operand (K or V)
+constexpr int kWarpLoader0 = 8, kWarpMma = 12;
 constexpr int kBlockKeys = 128;
 constexpr int kD = 128;
 constexpr int kTileBytes = 128 * kD * 2;        // one 128 x 128 bf16 operand tile: 32 KB
 constexpr int kHalfBytes = kTileBytes / 2;      // 64 head_dim columns of it
-constexpr int kKvStages = 3;
+constexpr int kKStages = 3, kVStages = 2;
 constexpr float kRescaleThreshold = 8.0f;       // log2 units
 
 // shared-memory map (offsets from the 1024-aligned base)
-constexpr int kOffQ = 0;
-constexpr int kOffK = kOffQ + kTileBytes;
-constexpr int kOffV = kOffK + kKvStages * kTileBytes;
-constexpr int kOffBar = kOffV + kKvStages * kTileBytes;
+constexpr int kOffQ = 0;                                    // Q_A, Q_B
+constexpr int kOffK = kOffQ + 2 * kTileBytes;
+constexpr int kOffV = kOffK + kKStages * kTileBytes;
+constexpr int kOffBar = kOffV + kVStages * kTileBytes;
 enum {
   BAR_Q = 0,
-  BAR_K_FULL = 1,                      // [kKvStages]
-  BAR_K_EMPTY = BAR_K_FULL + kKvStages,
-  BAR_V_FULL = BAR_K_EMPTY + kKvStages,
-  BAR_V_EMPTY = BAR_V_FULL + kKvStages,
-  BAR_V_FIXED = BAR_V_EMPTY + kKvStages,
-  BAR_S_FULL = BAR_V_FIXED + 1,        // [2]
-  BAR_P_FULL = BAR_S_FULL + 2,         // [2]
-  BAR_O_FULL = BAR_P_FULL + 2,
-  BAR_COUNT = BAR_O_FULL + 1
+  BAR_K_FULL = 1,                         // [kKStages]
+  BAR_K_EMPTY = BAR_K_FULL + kKStages,    // [kKStages]
+  BAR_V_FULL = BAR_K_EMPTY + kKStages,    // [kVStages]
+  BAR_V_EMPTY = BAR_V_FULL + kVStages,    // [kVStages]
+  BAR_S_FULL = BAR_V_EMPTY + kVStages,    // [2] per tile
+  BAR_P_FULL = BAR_S_FULL + 2,            // [2] per tile
+  BAR_O_FULL = BAR_P_FULL + 2,            // [2] per tile
+  BAR_COUNT = BAR_O_FULL + 2
 };
 constexpr int kOffMisc = kOffBar + BAR_COUNT * 8;   // tmem base address, dead flag
 constexpr int kSmemBytes = kOffMisc + 16 + 1024;
+static_assert(kSmemBytes <= 232448, "exceeds the shared memory one CTA can opt into");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -136,14 +142,27 @@ __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) |
          ((128u >> 4) << 24);
 }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+  // src_bytes == 0 writes 16 zero bytes and reads nothing
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
 __global__ void __launch_bounds__(kPfThreads, 1)
-prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap kv_map,
-               const __grid_constant__ CUtensorMap q_map) {
+prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem = smem_raw + (base - smem_u32(smem_raw));
@@ -152,31 +171,35 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap kv_map,
   auto bar = [&](int i) { return bar0 + (uint32_t)i * 8u; };
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);  // [0] tmem base, [1] dead
 
-  const WorkItem it = s.items[blockIdx.x];
-  const int kv_head = blockIdx.y;
+  const WorkItem it = s.items[blockIdx.y];   // grid = (KV heads, items): every head of a heavy item starts early
+  const int kv_head = blockIdx.x;
   const int G = s.Hq / s.Hkv;
   const int ctx = s.row_ctx[it.row];
-  const int q_len = s.row_qlen[it.row];
   const int tok0 = s.row_tok0[it.row];
-  const int tile_tok = it.q_begin;                     // first token of the tile (inside the row)
-  const int k_end = it.k_end;
-  const int nb = (k_end + kBlockKeys - 1) / kBlockKeys;
-  const bool fix_last = (k_end % kBlockKeys) != 0;
+  // tile A: tokens [q_begin, q_begin + cnt_a), tile B: the cnt_b tokens after them (maybe none)
+  const int tile_tokens = 128 / G;
+  const int cnt_a = min(it.q_count, tile_tokens), cnt_b = it.q_count - cnt_a;
+  const int k_end_a = ctx + it.q_begin + cnt_a, k_end_b = k_end_a + cnt_b;
+  const int nb_a = (k_end_a + kBlockKeys - 1) / kBlockKeys;
+  const int nb_b = cnt_b > 0 ? (k_end_b + kBlockKeys - 1) / kBlockKeys : 0;
+  const int nb = max(nb_a, nb_b);                       // K/V blocks this CTA streams
+  const int k_end = max(k_end_a, k_end_b);
 
   if (tid == 0) {
     misc[1] = 0;
     for (int i = 0; i < BAR_COUNT; ++i) {
       const bool softmax_arrives = i >= BAR_P_FULL && i < BAR_P_FULL + 2;
-      mbar_init(bar(i), softmax_arrives ? 128 : 1);
+      const bool loaders_arrive = (i >= BAR_K_FULL && i < BAR_K_FULL + kKStages) ||
+                                  (i >= BAR_V_FULL && i < BAR_V_FULL + kVStages);
+      mbar_init(bar(i), softmax_arrives ? 128 : loaders_arrive ? kLoaderThreads : 1);
     }
     mbar_init_fence();
   }
-  if (warp == 5) tmem_alloc(base + kOffMisc, 512);
+  if (warp == kWarpMma) tmem_alloc(base + kOffMisc, 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = misc[0];
-  const uint32_t tS0 = tmem, tO = tmem + 256;          // S buffers at columns 0 and 128, O at 256
 
   auto give_up = [&]() {
     if (misc[1] == 0) {
@@ -188,204 +211,270 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap kv_map,
     if (!mbar_wait(bar(i), parity, misc[1] ? 2000 : kWaitCycles)) give_up();
   };
 
-  if (warp == 4) {
-    // ------------------------------------------------------------------ TMA producer
+  if (warp >= kWarpLoader0 && warp < kWarpLoader0 + 4) {
+    // ------------------------------------------------------------------ K/V loaders
+    // 64 threads per operand copy each 128-key tile with 16-byte cp.async straight into the
+    // 128-byte-swizzled operand layout. (TMA is not used for K/V: with 16-token pages every
+    // tensor copy is only 2 KB, and the copy engine's per-request cost would bound the kernel.)
+    // K and V are two independent pipelines. A tile is announced at the start of a later
+    // iteration of its own loader, before that iteration waits for a free stage, so the
+    // announcement depends only on the copy having landed.
+    const int kv = (warp - kWarpLoader0) >> 1;               // 0: K, 1: V
+    const int t = tid - 256 - kv * kLoaderThreads;           // 0..63 inside the group
+    const int col16 = t & 15, rb = t >> 4;                   // chunk col16 of rows rb + 4 h + 8 i
     const int32_t* table_row = s.table + (size_t)s.row_slot[it.row] * s.max_pages_per_req;
-    if (lane == 0) {
-      tma_prefetch_desc(&kv_map);
+    if (kv == 0 && t == 0) {
       tma_prefetch_desc(&q_map);
-      mbar_expect_tx(bar(BAR_Q), kTileBytes);
-      tma_load_4d(base + kOffQ, &q_map, bar(BAR_Q), 0, 0, kv_head, tok0 + tile_tok);
-      tma_load_4d(base + kOffQ + kHalfBytes, &q_map, bar(BAR_Q), 64, 0, kv_head, tok0 + tile_tok);
-    }
-    for (int j = 0; j < nb; ++j) {
-      const int st = j % kKvStages;
-      const uint32_t ph = (j / kKvStages) & 1;
-      const int key0 = j * kBlockKeys;
-      const int n_pg = min(8, (k_end - key0 + kPageSize - 1) / kPageSize);
-      int page = 0;
-      if (lane < n_pg) {
-        page = table_row[(key0 >> 4) + lane];
-        if ((unsigned)page >= (unsigned)s.n_pages) {
-          atomicOr(s.status, TS_DEV_BAD_PAGE);
-          page = s.n_pages;                            // out of range: the copy delivers zeros
-        }
+      mbar_expect_tx(bar(BAR_Q), (cnt_b > 0 ? 2 : 1) * kTileBytes);
+      const int ta = tok0 + it.q_begin;
+      tma_load_4d(base + kOffQ, &q_map, bar(BAR_Q), 0, 0, kv_head, ta);
+      tma_load_4d(base + kOffQ + kHalfBytes, &q_map, bar(BAR_Q), 64, 0, kv_head, ta);
+      if (cnt_b > 0) {
+        tma_load_4d(base + kOffQ + kTileBytes, &q_map, bar(BAR_Q), 0, 0, kv_head, ta + tile_tokens);
+        tma_load_4d(base + kOffQ + kTileBytes + kHalfBytes, &q_map, bar(BAR_Q), 64, 0, kv_head, ta + tile_tokens);
       }
-      const int my_page = __shfl_sync(0xffffffffu, page, lane >> 1);
-      for (int kv = 0; kv < 2; ++kv) {
-        const int full = kv ? BAR_V_FULL : BAR_K_FULL, empty = kv ? BAR_V_EMPTY : BAR_K_EMPTY;
-        if (j >= kKvStages) wait(empty + st, ph ^ 1);
-        __syncwarp();
-        if (!misc[1]) {
-          if (lane == 0) mbar_expect_tx(bar(full + st), n_pg * 2 * kPageSize * kD);
-          if (lane < 2 * n_pg) {
-            const uint32_t dst = base + (kv ? kOffV : kOffK) + st * kTileBytes + (lane & 1) * kHalfBytes +
-                                 (lane >> 1) * (kPageSize * 128);
-            tma_load_5d(dst, &kv_map, bar(full + st), (lane & 1) * 64, 0, kv_head, kv, my_page);
+    }
+    const int stages = kv ? kVStages : kKStages;
+    const int lag = stages - 1;                              // tiles in flight besides the announced one
+    const int full = kv ? BAR_V_FULL : BAR_K_FULL, empty = kv ? BAR_V_EMPTY : BAR_K_EMPTY;
+    const uint32_t tile0 = base + (kv ? kOffV : kOffK);
+    const size_t head_off = ((size_t)kv * s.Hkv + kv_head) * kPageSize * kD + col16 * 8;
+    const size_t page_stride = (size_t)2 * s.Hkv * kPageSize * kD;
+    auto fetch_pages = [&](int j, int (&pg)[8]) {
+#pragma unroll
+      for (int p = 0; p < 8; ++p) {
+        const int key = j * kBlockKeys + p * kPageSize;
+        int page = -1;
+        if (key < k_end) {
+          page = table_row[key >> 4];
+          if ((unsigned)page >= (unsigned)s.n_pages) {
+            atomicOr(s.status, TS_DEV_BAD_PAGE);
+            page = -1;
           }
         }
+        pg[p] = page;
       }
-      if (j == nb - 1 && fix_last) {
-        // rows of the V block past the last visible key hold stale bits: clear them, so that
-        // a zero weight cannot meet a NaN
-        wait(BAR_V_FULL + st, ph);
-        const int valid = k_end - key0;
-        unsigned char* vb = smem + kOffV + st * kTileBytes;
-        for (int i = lane; i < (kBlockKeys - valid) * 16; i += 32) {
-          const int r = valid + i / 16, c = i % 16;
-          *reinterpret_cast<uint4*>(vb + (c >> 3) * kHalfBytes + r * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
+    };
+    auto announce = [&](int tile, int pending_allowed) {
+      if (pending_allowed >= 1) cp_async_wait<1>(); else cp_async_wait<0>();
+      fence_proxy_async();
+      mbar_arrive(bar(full + tile % stages));
+    };
+    int pg[8];
+    fetch_pages(0, pg);
+    for (int j = 0; j < nb; ++j) {
+      const int st = j % stages;
+      const int key0 = j * kBlockKeys;
+      int pg_next[8];
+      if (j + 1 < nb) fetch_pages(j + 1, pg_next);
+      if (j >= lag) announce(j - lag, lag - 1);              // K: tile j-2 (j-1 in flight); V: tile j-1
+      if (j >= stages) wait(empty + st, ((j / stages) & 1) ^ 1);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int r0 = rb + 4 * h;
+        const uint32_t dst = tile0 + st * kTileBytes +
+                             (uint32_t)((col16 >> 3) * kHalfBytes + r0 * 128 + (((col16 & 7) ^ r0) << 4));
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int row = r0 + 8 * i;
+          const int page = pg[i >> 1];
+          const bool valid = page >= 0 && key0 + row < k_end;   // rows past the last key are zero-filled
+          const uint16_t* src = valid ? s.pool + (size_t)page * page_stride + head_off + (row & 15) * kD : s.pool;
+          cp_async16(dst + i * 1024, src, valid ? 16 : 0);
         }
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_V_FIXED));
       }
+      cp_async_commit();
+#pragma unroll
+      for (int p = 0; p < 8; ++p) pg[p] = pg_next[p];
     }
-  } else if (warp == 5) {
+    // the last `lag` tiles (fewer when the item is short) have not been announced yet
+    for (int tile = max(0, nb - lag); tile < nb; ++tile) announce(tile, nb - 1 - tile);
+  } else if (warp == kWarpMma) {
     // ------------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
-      auto issue_qk = [&](int j) {
-        const int st = j % kKvStages;
-        wait(BAR_K_FULL + st, (j / kKvStages) & 1);
-        tc_fence_after();
-        if (!misc[1]) {
-          const uint32_t d = tS0 + (j & 1) * 128;
+      // descriptors differ only in their start-address field (16-byte units in the low bits)
+      const uint64_t q_desc0 = smem_desc(base + kOffQ, 0, 1024);
+      const uint64_t k_desc0 = smem_desc(base + kOffK, 0, 1024);
+      const uint64_t v_desc0 = smem_desc(base + kOffV, kHalfBytes, 1024);
+      auto issue_qk = [&](int x, int j) {          // S_x = Q_x K(j)^T
+        const uint64_t q_desc = q_desc0 + (uint64_t)((x * kTileBytes) >> 4);
+        const uint64_t k_desc = k_desc0 + (uint64_t)(((j % kKStages) * kTileBytes) >> 4);
 #pragma unroll
-          for (int ks = 0; ks < kD / 16; ++ks) {
-            const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-            mma_ss(d, smem_desc(base + kOffQ + off, 0, 1024),
-                   smem_desc(base + kOffK + st * kTileBytes + off, 0, 1024), idesc_qk, ks > 0);
-          }
-          tc_commit(bar(BAR_K_EMPTY + st));
-          tc_commit(bar(BAR_S_FULL + (j & 1)));
+        for (int ks = 0; ks < kD / 16; ++ks) {
+          const uint64_t off = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+          mma_ss(tmem + x * 128, q_desc + off, k_desc + off, idesc_qk, ks > 0);
         }
+        tc_commit(bar(BAR_S_FULL + x));
       };
-      wait(BAR_Q, 0);
-      issue_qk(0);
-      for (int j = 0; j < nb; ++j) {
-        if (j + 1 < nb) issue_qk(j + 1);
-        const int st = j % kKvStages;
-        wait(BAR_P_FULL + (j & 1), (j >> 1) & 1);
-        wait(BAR_V_FULL + st, (j / kKvStages) & 1);
-        if (j == nb - 1 && fix_last) wait(BAR_V_FIXED, 0);
-        tc_fence_after();
-        if (!misc[1]) {
-          const uint32_t p = tS0 + (j & 1) * 128;      // P(j): bf16 pairs in the first 64 columns of S(j)
+      auto issue_pv = [&](int x, int j) {          // O_x += P_x V(j)
+        const uint64_t v_desc = v_desc0 + (uint64_t)(((j % kVStages) * kTileBytes) >> 4);
 #pragma unroll
-          for (int kk = 0; kk < kBlockKeys / 16; ++kk) {
-            mma_ts(tO, p + kk * 8, smem_desc(base + kOffV + st * kTileBytes + kk * 2048, kHalfBytes, 1024),
-                   idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+        for (int kk = 0; kk < kBlockKeys / 16; ++kk)
+          mma_ts(tmem + 256 + x * 128, tmem + x * 128 + kk * 8, v_desc + (uint64_t)((kk * 2048) >> 4), idesc_pv,
+                 (j > 0 || kk > 0) ? 1u : 0u);
+        tc_commit(bar(BAR_O_FULL + x));
+      };
+      // Order: both Q K^T of block 0; then per block, for tile A then tile B:
+      // P V of block j followed at once by Q K^T of block j+1 of the same tile, so that the
+      // tile's warpgroup gets its next scores while the pipe turns to the other tile.
+      wait(BAR_Q, 0);
+      wait(BAR_K_FULL + 0, 0);
+      tc_fence_after();
+      if (!misc[1]) {
+        if (nb_a > 0) issue_qk(0, 0);
+        if (nb_b > 0) issue_qk(1, 0);
+        tc_commit(bar(BAR_K_EMPTY + 0));
+      }
+      for (int j = 0; j < nb; ++j) {
+        const bool next = j + 1 < nb;
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          const int nbx = x ? nb_b : nb_a;
+          if (j < nbx) {
+            wait(BAR_P_FULL + x, j & 1);
+            if (x == 0 || j >= nb_a) wait(BAR_V_FULL + j % kVStages, (j / kVStages) & 1);
+            tc_fence_after();
+            if (!misc[1]) issue_pv(x, j);
           }
-          tc_commit(bar(BAR_V_EMPTY + st));
-          tc_commit(bar(BAR_O_FULL));
+          if (x == 1 && !misc[1]) tc_commit(bar(BAR_V_EMPTY + j % kVStages));   // both tiles are done with V(j)
+          if (next) {
+            if (x == 0 || j + 1 >= nb_a) wait(BAR_K_FULL + (j + 1) % kKStages, ((j + 1) / kKStages) & 1);
+            tc_fence_after();
+            if (j + 1 < nbx && !misc[1]) issue_qk(x, j + 1);
+            if (x == 1 && !misc[1]) tc_commit(bar(BAR_K_EMPTY + (j + 1) % kKStages));
+          }
         }
       }
     }
     __syncwarp();
-  } else if (warp < 4) {
-    // ---------------------------------------------------- softmax + epilogue (row = tid)
-    const int row = tid;
-    const int rows_used = (128 / G) * G;
-    const int tok = tile_tok + row / G;
-    const bool real = row < rows_used && tok < q_len;
-    const int lim = real ? ctx + tok + 1 : k_end;       // keys at positions >= lim are masked
-    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+  } else {
+    // ------------------------------------------ softmax + epilogue: thread = query row of tile x
+    const int x = warp >> 2;
+    const int row = (warp & 3) * 32 + lane;
+    const int nbx = x ? nb_b : nb_a;
+    const int cnt = x ? cnt_b : cnt_a;
+    const int tok = it.q_begin + x * tile_tokens + row / G;   // token inside the request row
+    const bool real = row / G < cnt && row < tile_tokens * G;
+    const int k_end_x = x ? k_end_b : k_end_a;
+    const int lim = real ? ctx + tok + 1 : k_end_x;           // keys at positions >= lim are masked
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + x * 128 + lane_addr, tO = tmem + 256 + x * 128 + lane_addr;
     float m_ref = -CUDART_INF_F, l = 0.f;
-    for (int j = 0; j < nb; ++j) {
-      const uint32_t tS = tS0 + (j & 1) * 128 + lane_addr;
-      wait(BAR_S_FULL + (j & 1), (j >> 1) & 1);
+    for (int j = 0; j < nbx; ++j) {
+      wait(BAR_S_FULL + x, j & 1);
       tc_fence_after();
-      float sv[4][32];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(sv[c], tS + c * 32);
-      tmem_ld_wait();
       const int key0 = j * kBlockKeys;
       const bool need_mask = key0 + kBlockKeys > lim;
+      // pass 1: row maximum of the raw scores (the scale is positive, so it commutes with max)
       float mx = -CUDART_INF_F;
-#pragma unroll
+#pragma unroll 1
       for (int c = 0; c < 4; ++c) {
+        float v[32];
+        tmem_ld32(v, tS + c * 32);
+        tmem_ld_wait();
+        if (need_mask) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float v = sv[c][i] * s.scale_log2;
-          if (need_mask && key0 + c * 32 + i >= lim) v = -CUDART_INF_F;
-          sv[c][i] = v;
-          mx = fmaxf(mx, v);
+          for (int i = 0; i < 32; ++i)
+            if (key0 + c * 32 + i >= lim) v[i] = -CUDART_INF_F;
         }
+        float m0 = v[0], m1 = v[1], m2 = v[2], m3 = v[3];   // four short chains instead of one long one
+#pragma unroll
+        for (int i = 4; i < 32; i += 4) {
+          m0 = fmaxf(m0, v[i]);
+          m1 = fmaxf(m1, v[i + 1]);
+          m2 = fmaxf(m2, v[i + 2]);
+          m3 = fmaxf(m3, v[i + 3]);
+        }
+        mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
       }
+      mx *= s.scale_log2;
       // lazy rescale: move the reference maximum only when it is exceeded by 2^threshold
       const bool move = mx > m_ref + kRescaleThreshold;   // first block: m_ref = -inf, so true
       float alpha = 1.f;
       if (move) {
-        alpha = exp2f(m_ref - mx);                        // 0 on the first block
+        alpha = ex2(m_ref - mx);                          // 0 on the first block
         m_ref = mx;
         l *= alpha;
       }
       if (j > 0 && __any_sync(0xffffffffu, move)) {
-        wait(BAR_O_FULL, (j - 1) & 1);                    // P V of block j-1 has landed in O
+        wait(BAR_O_FULL + x, (j - 1) & 1);                // P V of block j-1 has landed in O
         tc_fence_after();
-#pragma unroll
+#pragma unroll 1
         for (int c = 0; c < 4; ++c) {
           float ov[32];
-          tmem_ld32(ov, tO + lane_addr + c * 32);
+          tmem_ld32(ov, tO + c * 32);
           tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 32; ++i) ov[i] *= alpha;
-          tmem_st32(tO + lane_addr + c * 32, ov);
+          tmem_st32(tO + c * 32, ov);
         }
       }
-      float rs = 0.f;
-#pragma unroll
+      // pass 2: p = 2^(s*scale - m_ref), packed to bf16 over the part of S already consumed
+      const float neg_m = -m_ref;
+      float rs = 0.f, rs1 = 0.f;
+#pragma unroll 1
       for (int c = 0; c < 4; ++c) {
+        float v[32];
+        tmem_ld32(v, tS + c * 32);
+        tmem_ld_wait();
         uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          const float p0 = exp2f(sv[c][2 * i] - m_ref), p1 = exp2f(sv[c][2 * i + 1] - m_ref);
-          rs += p0 + p1;
+          float p0 = ex2(fmaf(v[2 * i], s.scale_log2, neg_m));
+          float p1 = ex2(fmaf(v[2 * i + 1], s.scale_log2, neg_m));
+          if (need_mask) {
+            if (key0 + c * 32 + 2 * i >= lim) p0 = 0.f;
+            if (key0 + c * 32 + 2 * i + 1 >= lim) p1 = 0.f;
+          }
+          if (i & 1) rs1 += p0 + p1; else rs += p0 + p1;
           pk[i] = pack2(p0, p1);
         }
-        tmem_st16(tS + c * 16, pk);                        // P overwrites the part of S already consumed
+        tmem_st16(tS + c * 16, pk);       // columns [16c, 16c+16): scores there were read already
       }
+      rs += rs1;
       l += rs;
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(bar(BAR_P_FULL + (j & 1)));
+      mbar_arrive(bar(BAR_P_FULL + x));
     }
-    // epilogue: O / l -> bf16 -> global
-    wait(BAR_O_FULL, (nb - 1) & 1);
-    tc_fence_after();
-    const float inv = 1.f / l;
-    uint16_t* orow = s.out + ((size_t)(tok0 + tok) * s.Hq + kv_head * G + row % G) * kD;
+    if (nbx > 0) {
+      // epilogue: O / l -> bf16 -> global
+      wait(BAR_O_FULL + x, (nbx - 1) & 1);
+      tc_fence_after();
+      const float inv = 1.f / l;
+      uint16_t* orow = s.out + ((size_t)(tok0 + tok) * s.Hq + kv_head * G + row % G) * kD;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float ov[32];
+        tmem_ld32(ov, tO + c * 32);
+        tmem_ld_wait();
+        if (real) {
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      float ov[32];
-      tmem_ld32(ov, tO + lane_addr + c * 32);
-      tmem_ld_wait();
-      if (real) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint4 w;
-          w.x = pack2(ov[8 * i] * inv, ov[8 * i + 1] * inv);
-          w.y = pack2(ov[8 * i + 2] * inv, ov[8 * i + 3] * inv);
-          w.z = pack2(ov[8 * i + 4] * inv, ov[8 * i + 5] * inv);
-          w.w = pack2(ov[8 * i + 6] * inv, ov[8 * i + 7] * inv);
-          *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = w;
+          for (int i = 0; i < 4; ++i) {
+            uint4 w;
+            w.x = pack2(ov[8 * i] * inv, ov[8 * i + 1] * inv);
+            w.y = pack2(ov[8 * i + 2] * inv, ov[8 * i + 3] * inv);
+            w.z = pack2(ov[8 * i + 4] * inv, ov[8 * i + 5] * inv);
+            w.w = pack2(ov[8 * i + 6] * inv, ov[8 * i + 7] * inv);
+            *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = w;
+          }
         }
       }
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem, 512);
+  if (warp == kWarpMma) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace
 
-cudaError_t launch_prefill(const StepDevice& s, const CUtensorMap& kv_map, const CUtensorMap& q_map,
-                           cudaStream_t stream) {
+cudaError_t launch_prefill(const StepDevice& s, const CUtensorMap& q_map, cudaStream_t stream) {
   if (s.n_prefill_items <= 0) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
-  prefill_kernel<<<dim3(s.n_prefill_items, s.Hkv), kPfThreads, kSmemBytes, stream>>>(s, kv_map, q_map);
+  prefill_kernel<<<dim3(s.Hkv, s.n_prefill_items), kPfThreads, kSmemBytes, stream>>>(s, q_map);
   return cudaGetLastError();
 }
 

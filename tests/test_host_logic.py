@@ -163,7 +163,7 @@ def test_step_validation_launches_nothing():
     B.ts_destroy(h)
 
 
-def _check_plan(items, G, rows, tile_rows=128):
+def _check_plan(items, G, rows, tile_rows=256):
     """Every (packed query row, key) pair of the step is covered exactly once."""
     by_row = {}
     for it in items:
