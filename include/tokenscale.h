@@ -262,7 +262,7 @@ int ts_plan_step(ts_ctx* ctx, const ts_step* step, int32_t* items, int32_t items
  * 0, or a bit set of TS_DEV_* flags raised by kernels (they skip the offending access
  * instead of faulting).
  */
-enum { TS_DEV_BAD_PAGE = 1, TS_DEV_TIMEOUT = 2 };
+enum { TS_DEV_BAD_PAGE = 1, TS_DEV_TIMEOUT = 2, TS_DEV_BAD_INDEX = 4 };
 int ts_last_device_status(ts_ctx* ctx, void* cuda_stream, int32_t* status_out);
 
 /*

@@ -24,6 +24,7 @@ TS_ERR_WORKSPACE = -9
 TS_STEP_KEEP_LEN = 1
 TS_DEV_BAD_PAGE = 1
 TS_DEV_TIMEOUT = 2
+TS_DEV_BAD_INDEX = 4
 
 _i32p = ctypes.POINTER(ctypes.c_int32)
 

@@ -357,6 +357,7 @@ int sync_tables(ts_ctx* c, const ts_step* st, cudaStream_t stream) {
     if (rc != TS_OK) return rc;
     char* ws = (char*)c->cfg.workspace;
     TS_CUDA(c, ts::launch_table_update((int32_t*)(ws + c->L.off_table), c->cfg.max_pages_per_req,
+                                       c->cfg.max_requests, (int32_t*)(ws + c->L.off_status),
                                        (const TableDelta*)(ws + c->L.off_delta), (int)n, stream));
     ++c->cnt.kernel_launches;
     at += n;
@@ -414,6 +415,7 @@ void fill_device(ts_ctx* c, const ts_step* st, int64_t n_tokens, ts::StepDevice*
   d->D = c->cfg.head_dim;
   d->n_pages = c->cfg.n_pages;
   d->max_pages_per_req = c->cfg.max_pages_per_req;
+  d->max_requests = c->cfg.max_requests;
   d->scale_log2 = c->scale * 1.4426950408889634f;
 }
 

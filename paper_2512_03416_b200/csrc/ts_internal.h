@@ -63,13 +63,13 @@ struct StepDevice {
   // shape
   int32_t n_rows, n_tokens, n_items, n_combines;
   int32_t n_prefill_items;  // items[0, n_prefill_items) are prefill tiles, the rest decode splits
-  int32_t Hq, Hkv, D, n_pages, max_pages_per_req;
+  int32_t Hq, Hkv, D, n_pages, max_pages_per_req, max_requests;
   float scale_log2;        // softmax scale * log2(e)
 };
 
 // Launchers. Each enqueues on `stream` and returns the launch's cudaError_t.
-cudaError_t launch_table_update(int32_t* table, int max_pages_per_req, const TableDelta* deltas,
-                                int n_deltas, cudaStream_t stream);
+cudaError_t launch_table_update(int32_t* table, int max_pages_per_req, int max_requests, int32_t* status,
+                                const TableDelta* deltas, int n_deltas, cudaStream_t stream);
 cudaError_t launch_kv_append(const StepDevice& s, cudaStream_t stream);
 cudaError_t launch_attention(const StepDevice& s, cudaStream_t stream);
 cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream);

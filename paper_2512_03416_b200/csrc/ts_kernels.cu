@@ -57,9 +57,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // ------------------------------------------------------------------------------ small kernels
-__global__ void table_update_kernel(int32_t* table, int width, const TableDelta* deltas, int n) {
+__global__ void table_update_kernel(int32_t* table, int width, int max_requests, int32_t* status,
+                                    const TableDelta* deltas, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) table[(size_t)deltas[i].slot * width + deltas[i].index] = deltas[i].page;
+  if (i >= n) return;
+  const TableDelta d = deltas[i];
+  if ((unsigned)d.slot >= (unsigned)max_requests || (unsigned)d.index >= (unsigned)width) {
+    atomicOr(status, TS_DEV_BAD_INDEX);        // never expected: the host builds these records
+    return;
+  }
+  table[(size_t)d.slot * width + d.index] = d.page;
 }
 
 // One thread per 16-byte chunk of new K or V: chunk -> (token, K|V, head, 8 elements).
@@ -82,7 +89,12 @@ __global__ void kv_append_kernel(StepDevice s) {
       if (s.row_tok0[mid] <= tok) lo = mid; else hi = mid;
     }
     const int t = s.row_ctx[lo] + (tok - s.row_tok0[lo]);
-    const int page = s.table[(size_t)s.row_slot[lo] * s.max_pages_per_req + (t >> 4)];
+    const int slot = s.row_slot[lo];
+    if ((unsigned)slot >= (unsigned)s.max_requests || (unsigned)(t >> 4) >= (unsigned)s.max_pages_per_req) {
+      atomicOr(s.status, TS_DEV_BAD_INDEX);
+      continue;
+    }
+    const int page = s.table[(size_t)slot * s.max_pages_per_req + (t >> 4)];
     if ((unsigned)page >= (unsigned)s.n_pages) {
       atomicOr(s.status, TS_DEV_BAD_PAGE);
       continue;
@@ -97,15 +109,19 @@ __global__ void kv_append_kernel(StepDevice s) {
 __global__ void combine_kernel(StepDevice s) {
   const CombineItem c = s.combines[blockIdx.x];
   const int h = blockIdx.y, d = threadIdx.x;
+  // the loads of different splits are independent: unrolling keeps several of them in flight
+  const float* ml = s.part_ml + ((size_t)c.first_partial * s.Hq + h) * 2;
+  const float* pa = s.part_acc + ((size_t)c.first_partial * s.Hq + h) * s.D + d;
+  const size_t ml_stride = (size_t)s.Hq * 2, pa_stride = (size_t)s.Hq * s.D;
   float m = -CUDART_INF_F;
-  for (int i = 0; i < c.n_splits; ++i)
-    m = fmaxf(m, s.part_ml[((size_t)(c.first_partial + i) * s.Hq + h) * 2]);
+#pragma unroll 8
+  for (int i = 0; i < c.n_splits; ++i) m = fmaxf(m, ml[i * ml_stride]);
   float l = 0.f, acc = 0.f;
+#pragma unroll 8
   for (int i = 0; i < c.n_splits; ++i) {
-    const size_t ph = (size_t)(c.first_partial + i) * s.Hq + h;
-    const float w = exp2f(s.part_ml[ph * 2] - m);
-    l += w * s.part_ml[ph * 2 + 1];
-    acc += w * s.part_acc[ph * s.D + d];
+    const float w = exp2f(ml[i * ml_stride] - m);
+    l += w * ml[i * ml_stride + 1];
+    acc += w * pa[i * pa_stride];
   }
   s.out[((size_t)c.token * s.Hq + h) * s.D + d] = __bfloat16_as_ushort(__float2bfloat16_rn(acc / l));
 }
@@ -393,10 +409,11 @@ cudaError_t launch_attention_d(const StepDevice& s, cudaStream_t stream) {
 
 }  // namespace
 
-cudaError_t launch_table_update(int32_t* table, int max_pages_per_req, const TableDelta* deltas,
-                                int n_deltas, cudaStream_t stream) {
+cudaError_t launch_table_update(int32_t* table, int max_pages_per_req, int max_requests, int32_t* status,
+                                const TableDelta* deltas, int n_deltas, cudaStream_t stream) {
   if (n_deltas <= 0) return cudaSuccess;
-  table_update_kernel<<<(n_deltas + 255) / 256, 256, 0, stream>>>(table, max_pages_per_req, deltas, n_deltas);
+  table_update_kernel<<<(n_deltas + 255) / 256, 256, 0, stream>>>(table, max_pages_per_req, max_requests, status,
+                                                                  deltas, n_deltas);
   return cudaGetLastError();
 }
 
@@ -563,6 +580,7 @@ extern "C" int ts_decode_attention_static(int32_t device, int32_t n_q_heads, int
   d.D = head_dim;
   d.n_pages = n_pages;
   d.max_pages_per_req = table_width;
+  d.max_requests = n_rows;
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
   d.scale_log2 = scale * 1.4426950408889634f;
   if (launch_attention(d, stream) != cudaSuccess) return TS_ERR_CUDA;

@@ -1,0 +1,148 @@
+"""Drives a Decoder through a TraceReplay (bursty arrivals on a Convertible Decoder).
+
+Every replay step becomes one ts_mixed_step: the live decode requests take one token each and at
+most one prefill task is absorbed, chunk by chunk (Sec. 3.4, Sec. 4.4). Requests are added, their
+pages grown and released through the library's own allocator, so block tables and page
+scattering arise the way they do in serving. No oracle code is imported here.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, List, Optional
+
+import numpy as np
+import torch
+
+from . import workloads as wl
+from .decoder import Decoder
+from .harness import to_dev
+
+
+@dataclass
+class PreparedStep:
+    index: int
+    adds: list
+    preload: list
+    frees: List[int]
+    req_ids: List[int]
+    q_len: List[int]
+    ctx_len: List[int]
+    q: Optional[torch.Tensor] = None       # device tensors of the step (None for an empty step)
+    k_new: Optional[torch.Tensor] = None
+    v_new: Optional[torch.Tensor] = None
+    out: Optional[torch.Tensor] = None
+    host: Optional[tuple] = None            # (q, k_new, v_new) bit patterns on the host, when kept
+
+    @property
+    def n_tokens(self) -> int:
+        return int(sum(self.q_len))
+
+    @property
+    def prefill_tokens(self) -> int:
+        return int(sum(t for t in self.q_len if t > 1))
+
+    @property
+    def decode_tokens(self) -> int:
+        return int(sum(1 for t in self.q_len if t == 1))
+
+
+class ReplayRunner:
+    def __init__(self, trace: wl.TraceReplay, seed: int = 50, device: int = 0, keep_host: bool = False,
+                 pool_pages: Optional[int] = None, nan_fill: bool = False, decode_split_tokens: int = 0):
+        self.trace = trace
+        self.shape = trace.shape
+        self.device = torch.device("cuda", device)
+        self.keep_host = keep_host
+        s = self.shape
+        self.bank = wl.ValueBank(seed, 1.0 / np.sqrt(s.D), log2_size=24)
+        self.steps: List[PreparedStep] = []
+        live_tokens, peak = {}, 0
+        warm_ctx: Dict[int, tuple] = {}
+        with torch.cuda.device(self.device):
+            for st in trace.steps():
+                for r, n in st.preload:                    # context of the requests in flight at step 0
+                    k = self.bank.take(n * s.Hkv * s.D).reshape(n, s.Hkv, s.D)
+                    v = self.bank.take(n * s.Hkv * s.D).reshape(n, s.Hkv, s.D)
+                    warm_ctx[r.req_id] = (k, v)
+                    live_tokens[r.req_id] = n
+                ps = PreparedStep(st.index, st.adds, st.preload, st.frees, [r[0] for r in st.rows],
+                                  [r[1] for r in st.rows], [r[2] for r in st.rows])
+                n = ps.n_tokens
+                if n:
+                    q, k, v = wl.replay_values(s, seed, n, self.bank)
+                    ps.q, ps.k_new, ps.v_new = to_dev(q, self.device), to_dev(k, self.device), to_dev(v, self.device)
+                    ps.out = torch.empty((n, s.Hq, s.D), dtype=torch.int16, device=self.device)
+                    if keep_host:
+                        ps.host = (q, k, v)
+                for rid, ql, ctx in st.rows:
+                    live_tokens[rid] = ctx + ql
+                pages_now = sum((t + s.P - 1) // s.P + 1 for t in live_tokens.values())
+                peak = max(peak, pages_now)
+                for rid in st.frees:
+                    live_tokens.pop(rid, None)
+                self.steps.append(ps)
+        self.warm_ctx = warm_ctx
+        n_pages = pool_pages or int(1.25 * peak) + 64
+        width = (trace.max_context + s.P - 1) // s.P + 1
+        self.dec = Decoder(s.Hq, s.Hkv, s.D, n_pages, trace.max_decodes + 8, width, chunk_size=trace.chunk_size,
+                           device=device, alloc_shuffle_seed=seed, nan_fill=nan_fill,
+                           decode_split_tokens=decode_split_tokens)
+        self.slot_of: Dict[int, int] = {}
+
+    # -------------------------------------------------------------------------------- one step
+    def begin_step(self, ps: PreparedStep) -> None:
+        """Host bookkeeping before the step: admit requests, load warm context, grow tables."""
+        for r in ps.adds:
+            self.slot_of[r.req_id] = self.dec.request_add(r.req_id, r.prompt_len, r.output_len)
+        for r, cached in ps.preload:
+            slot = self.slot_of[r.req_id]
+            k, v = self.warm_ctx[r.req_id]
+            self.dec.alloc_pages(slot, cached, for_prefill=True)
+            with torch.cuda.device(self.device):
+                self.dec.kv_append([slot], [cached], [0], to_dev(k, self.device), to_dev(v, self.device))
+        for rid, ql, ctx in zip(ps.req_ids, ps.q_len, ps.ctx_len):
+            self.dec.alloc_pages(self.slot_of[rid], ctx + ql, for_prefill=ql > 1)
+
+    def launch(self, ps: PreparedStep) -> None:
+        if not ps.req_ids:
+            return
+        with torch.cuda.device(self.device):
+            self.dec.mixed_step([self.slot_of[r] for r in ps.req_ids], ps.q_len, ps.ctx_len, ps.q, ps.k_new,
+                                ps.v_new, ps.out)
+
+    def end_step(self, ps: PreparedStep) -> None:
+        for rid in ps.frees:
+            self.dec.request_free(self.slot_of.pop(rid))
+
+    def tables(self, ps: PreparedStep) -> List[np.ndarray]:
+        return [self.dec.block_table(self.slot_of[r])[0] for r in ps.req_ids]
+
+    def step_work(self, ps: PreparedStep):
+        """(flops, bytes) of the step, same accounting as StepBatch.algorithmic_work."""
+        s = self.shape
+        keys, kv_tokens = 0.0, 0
+        for c, t in zip(ps.ctx_len, ps.q_len):
+            keys += t * c + t * (t + 1) / 2
+            kv_tokens += c + t
+        n = ps.n_tokens
+        return (4.0 * s.D * s.Hq * keys,
+                float(kv_tokens * s.kv_bytes_per_token + n * s.kv_bytes_per_token + 2 * n * s.Hq * s.D * 2))
+
+    def run(self, timed: bool = True):
+        """Runs every step in order; returns per-step milliseconds (CUDA events) when timed."""
+        ms = []
+        with torch.cuda.device(self.device):
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in self.steps] if timed else None
+            for i, ps in enumerate(self.steps):
+                self.begin_step(ps)
+                if timed:
+                    evs[i][0].record()
+                self.launch(ps)
+                if timed:
+                    evs[i][1].record()
+                self.end_step(ps)
+            torch.cuda.synchronize(self.device)
+            if timed:
+                ms = [a.elapsed_time(b) for a, b in evs]
+        return ms

@@ -296,7 +296,7 @@ class ReplayRequest:
 class ReplayStep:
     index: int
     adds: List[ReplayRequest]                 # requests that enter the instance before the step
-    preload: List[ReplayRequest]              # warm requests whose context must be loaded first
+    preload: List[tuple]                      # (warm request, tokens cached before step 0): load these first
     rows: List[tuple]                         # (req_id, q_len, ctx_len), decode rows first
     frees: List[int]                          # req_ids that complete with this step
 
@@ -368,7 +368,7 @@ class TraceReplay:
                 for r in self.warm_requests:
                     live.append(r)
                     adds.append(r)
-                    preload.append(r)
+                    preload.append((r, r.cached))      # the request objects advance as the replay runs
             while pending and pending[0].arrival_s <= now:
                 queue.append(pending.pop(0))
             n_live = len(live) + (1 if task is not None else 0)
