@@ -6,6 +6,10 @@
 One "step" is one pass of the whole path (table sync, KV append, attention over decode rows and
 prefill chunks, split combine) over one batch. Prints ONE JSON line on rank 0.
 N > 1 runs N independent replicas (the path has no exchange step): weak scaling.
+
+Workloads: config2 decode-only batch, config3 convertible-decoder burst (default, the mixed step
+the metric names), config4 chunked-prefill continuation, config5 bursty trace replay on a
+70B-shaped layer (there a step is one replay step and K is capped by the replay's 200 steps).
 """
 from __future__ import annotations
 
@@ -32,6 +36,7 @@ WORKLOADS = {
     "config2": (wl.config2, "decode-only batch, 8B-shaped layer (64 decode rows, ctx lognormal median 2048)"),
     "config3": (wl.config3, "convertible-decoder burst, 8B-shaped layer (64 decode rows + one fresh 2048-token prefill chunk)"),
     "config4": (wl.config4, "chunked-prefill continuation, 8B-shaped layer (128 decode rows + 4 chunks of 512 tokens)"),
+    "config5": (None, "bursty trace replay, 70B-shaped layer (200 steps, Gamma arrivals CV=4, <=256 decodes, one prefill task at a time)"),
 }
 
 
@@ -45,6 +50,33 @@ def load_peaks():
         except Exception:
             pass
     return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------ multi-process plumbing
+def dist_env():
+    return (int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Each replica draws its own batch; rank 0 keeps the documented seed."""
+    return base_seed + 1000 * rank
+
+
+def reduce_max(value: float, world: int, device=None) -> float:
+    """Max over ranks of a timing (every multi-GPU number is the slowest rank's)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(units_per_rank: float, world: int, seconds_max: float) -> float:
+    """Whole-job throughput: units all ranks processed over the slowest rank's time."""
+    return world * units_per_rank / seconds_max
 
 
 class ClockSampler(threading.Thread):
@@ -70,13 +102,8 @@ class ClockSampler(threading.Thread):
         if not self.ok:
             return
         nv = self.nv
-        names = {
-            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
-            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
-            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
-            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
-            getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
-        }
+        names = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+                 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
         while not self._stop_evt.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
@@ -159,12 +186,42 @@ class OracleLeg:
         return int(min(max(1, math.ceil(total / (rate * seconds))), max(1, b.n_tokens)))
 
 
+def replay_heavy_batch():
+    """The replay's heaviest kind of step as a static batch (what the oracle legs sample for config5):
+    192 decode rows with the replay's context mix plus one fresh 8192-token prefill chunk."""
+    rng = np.random.Generator(np.random.Philox(5))
+    ctx = wl._lognormal_lengths(rng, 1024, 1.0, 16, 8192, 192) + wl._lognormal_lengths(rng, 256, 1.0, 1, 2048, 192) // 2
+    ctx = np.concatenate([ctx, [0]]).astype(np.int32)
+    ql = np.concatenate([np.ones(192, np.int32), [8192]]).astype(np.int32)
+    return wl.make_batch("config5_heavy_step", wl.LLAMA70B, ctx, ql, seed=105, chunk_size=8448)
+
+
+def make_static_batch(workload: str, rank: int):
+    if workload == "config5":
+        return replay_heavy_batch()
+    make = WORKLOADS[workload][0]
+    return make(seed=rank_seed(make.__defaults__[0], rank))
+
+
+def cpu_baseline_leg(batch, target_s: float = 10.0):
+    leg = OracleLeg(batch)
+    stride = leg.stride_for(target_s)
+    sel = oracle_sample(batch, stride)
+    t, reps = 0.0, 0
+    while t < target_s * 0.6 and reps < 64:          # repeat small workloads up to a few seconds of CPU work
+        t += leg.run(sel)
+        reps += 1
+    return {"value": reps * len(sel) / t, "unit": UNIT, "cores": leg.cores, "kind": "oracle",
+            "sample": f"every {stride}th decode row and every {stride}th prefill token of {batch.name} "
+                      f"({len(sel)} of {batch.n_tokens} tokens), repeated {reps}x, {t:.1f} s"}
+
+
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
+    world, rank, _ = dist_env()
     if rank != 0:
         return
-    make, desc = WORKLOADS[args.workload]
-    batch = make()
+    desc = WORKLOADS[args.workload][1]
+    batch = make_static_batch(args.workload, 0)
     leg = OracleLeg(batch)
     budget = 150.0 / max(1, args.steps + args.warmup)
     stride = leg.stride_for(budget)
@@ -176,7 +233,8 @@ def run_reference(args):
         t += leg.run(sel)
     per_step = t / max(1, args.steps)
     value = len(sel) / per_step
-    sample = f"every {stride}th decode row and every {stride}th prefill token ({len(sel)} of {batch.n_tokens} tokens) per step"
+    sample = (f"every {stride}th decode row and every {stride}th prefill token of {batch.name} "
+              f"({len(sel)} of {batch.n_tokens} tokens) per step")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
@@ -188,33 +246,39 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------- our arm
-def run_ours(args):
-    import torch
-    import torch.distributed as dist
+def rooflines(peaks, peak_kind, flops, byts, dec_bytes, pf_flops, step_ms, prof):
+    steps = max(1, prof["steps"])
+    dec_ms, pf_ms = prof["decode_ms"] / steps, prof["prefill_ms"] / steps
+    t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
+    t_tc = flops / (peaks["bf16_tflops"] * 1e12)
+    # the dominant kernel: decode attention (HBM) unless the prefill kernel takes longer (tensor)
+    if dec_ms >= pf_ms:
+        ach = dec_bytes / (dec_ms * 1e-3) / 1e9 if dec_ms > 0 else 0.0
+        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"], "traffic": None, "kernel": "decode_kernel", "kernel_ms": dec_ms}
+    else:
+        ach = pf_flops / (pf_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops"], "traffic": None, "kernel": "prefill_kernel", "kernel_ms": pf_ms}
+    roof.update({"peak_source": f"of {peak_kind}", "decode_ms": dec_ms, "prefill_ms": pf_ms,
+                 "append_ms": prof["append_ms"] / steps, "combine_ms": prof["combine_ms"] / steps,
+                 "decode_GBps": dec_bytes / (dec_ms * 1e-3) / 1e9 if dec_ms > 0 else None,
+                 "prefill_TFLOPs": pf_flops / (pf_ms * 1e-3) / 1e12 if pf_ms > 0 else None})
+    t_roof = max(t_hbm, t_tc)
+    step_roof = {"t_roof_us": t_roof * 1e6, "t_hbm_us": t_hbm * 1e6, "t_tensor_us": t_tc * 1e6,
+                 "frac": t_roof / (step_ms * 1e-3), "flops": flops, "bytes": byts,
+                 "frac_nominal": max(byts / 8e12, flops / 2.25e15) / (step_ms * 1e-3)}
+    return roof, step_roof
 
+
+def run_static(args, world, rank, local, barrier):
+    import torch
     from paper_2512_03416_b200.harness import LoadedBatch
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    make, desc = WORKLOADS[args.workload]
-    batch = make(seed=make.__defaults__[0] + 1000 * rank) if rank else make()
+    batch = make_static_batch(args.workload, rank)
     lb = LoadedBatch(batch, device=local, nan_fill=False)
-    flops, byts = batch.algorithmic_work()
-    peaks, peak_kind = load_peaks()
+    s = batch.shape
     K, W = args.steps, max(args.warmup, 3)
-
     for _ in range(W):
         lb.step_repeatable()
     barrier()
@@ -229,46 +293,21 @@ def run_ours(args):
     e1.record()
     barrier()
     clocks = sampler.stop()
-    ms_total = e0.elapsed_time(e1)
-    v1 = lb.dec.velocity()
-    launches = int(v1["kernel_launches"] - v0["kernel_launches"])
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-    ms_step = ms_total / K
+    ms_step = reduce_max(e0.elapsed_time(e1), world, "cuda") / K
+    launches = int(lb.dec.velocity()["kernel_launches"] - v0["kernel_launches"])
     tokens = batch.n_tokens
-    value = world * tokens / (ms_step * 1e-3)
 
-    # per-kernel device time (separate pass: the extra events perturb the step a little)
-    Kp = min(K, 300)
-    lb.dec.profile_enable(True)
-    for _ in range(Kp):
+    lb.dec.profile_enable(True)                       # separate pass: the extra events cost a little
+    for _ in range(min(K, 300)):
         lb.step_repeatable()
     prof = lb.dec.profile_read()
     lb.dec.profile_enable(False)
-    attn_ms = prof["attention_ms"] / max(1, prof["steps"])
-    s = batch.shape
-    kv_tokens = int((batch.ctx_len + batch.q_len).sum())
-    attn_bytes = kv_tokens * s.kv_bytes_per_token + 2 * tokens * s.Hq * s.D * 2
-    t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
-    t_tc = flops / (peaks["bf16_tflops"] * 1e12)
-    hbm_bound = t_hbm >= t_tc
-    if hbm_bound:
-        achieved = attn_bytes / (attn_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": None}
-    else:
-        achieved = flops / (attn_ms * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": achieved / peaks["bf16_tflops"], "traffic": None}
-    roofline.update({"kernel": "attention_kernel", "kernel_ms": attn_ms, "peak_source": f"of {peak_kind}",
-                     "append_ms": prof["append_ms"] / max(1, prof["steps"]),
-                     "combine_ms": prof["combine_ms"] / max(1, prof["steps"])})
-    t_roof = max(t_hbm, t_tc)
-    step_roofline = {"t_roof_us": t_roof * 1e6, "t_hbm_us": t_hbm * 1e6, "t_tensor_us": t_tc * 1e6,
-                     "frac": t_roof / (ms_step * 1e-3), "flops": flops, "bytes": byts,
-                     "frac_nominal_8TBs": max(byts / 8e12, flops / 2.25e15) / (ms_step * 1e-3)}
+
+    flops, byts = batch.algorithmic_work()
+    dec = batch.q_len == 1
+    dec_bytes = float(((batch.ctx_len[dec] + 1) * s.kv_bytes_per_token).sum() + 2 * dec.sum() * s.Hq * s.D * 2)
+    pf_flops = 4.0 * s.D * s.Hq * float(sum(t * c + t * (t + 1) / 2 for c, t in
+                                            zip(batch.ctx_len[~dec].tolist(), batch.q_len[~dec].tolist())))
 
     # end to end: host buffers in, host buffer out, through ts_mixed_step_host
     Ke = min(K, 300)
@@ -284,38 +323,149 @@ def run_ours(args):
     for _ in range(Ke):
         lb.dec.mixed_step_host(lb.slots, ql, cl, hq, hk, hv, ho, keep_len=True)
     torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e = {"value": world * tokens / (e2e_s / Ke), "unit": UNIT,
+    e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
+    e2e = {"value": aggregate_value(tokens, world, e2e_s / Ke), "unit": UNIT,
            "h2d_bytes_per_step": int(hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2),
            "d2h_bytes_per_step": int(ho.numel() * 2), "steps": Ke, "ms_per_step": e2e_s / Ke * 1e3}
+    kv_tokens = int((batch.ctx_len + batch.q_len).sum())
+    cfg = {"decode_rows": batch.decode_tokens, "prefill_tokens": batch.prefill_tokens, "kv_tokens": kv_tokens,
+           "l2": "inputs larger than L2 (KV working set %.2f GB)" % (kv_tokens * s.kv_bytes_per_token / 1e9)}
+    return dict(batch=batch, ms_step=ms_step, tokens=tokens, prefill_tokens=batch.prefill_tokens,
+                decode_tokens=batch.decode_tokens, launches=launches, clocks=clocks, prof=prof, flops=flops,
+                byts=byts, dec_bytes=dec_bytes, pf_flops=pf_flops, e2e=e2e, cfg=cfg, steps=K, warmup=W, extra={})
 
+
+def run_replay(args, world, rank, local, barrier):
+    """config5: the 200-step bursty replay. Every step is issued once, in order (the state evolves);
+    warm-up is a full untimed replay on a fresh instance."""
+    import torch
+    from paper_2512_03416_b200.replay import ReplayRunner
+
+    K = min(args.steps, 200)
+    seed = rank_seed(5, rank)
+
+    def fresh(keep_host=False):
+        return ReplayRunner(wl.TraceReplay(seed=seed, n_steps=K), seed=seed + 45, device=local, keep_host=keep_host)
+
+    warm = fresh()
+    warm.run(timed=False)                              # warm-up: every launch shape once
+    warm.dec.close()
+    del warm
+    run = fresh()
+    run.start()                                        # requests in flight at step 0: context resident before timing
+    s = run.shape
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    step_ms = run.run(timed=True)
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = reduce_max(e0.elapsed_time(e1), world, "cuda")
+    launches = int(run.dec.velocity()["kernel_launches"])
+    tokens = sum(ps.n_tokens for ps in run.steps)
+    pf_tok = sum(ps.prefill_tokens for ps in run.steps)
+    dec_tok = sum(ps.decode_tokens for ps in run.steps)
+    work = [run.step_work(ps) for ps in run.steps]
+    flops, byts = sum(w[0] for w in work), sum(w[1] for w in work)
+    peaks, _ = load_peaks()
+    t_roof = [max(w[1] / (peaks["hbm_gbs"] * 1e9), w[0] / (peaks["bf16_tflops"] * 1e12)) for w in work]
+    run.dec.close()
+
+    # per-kernel times: one more replay with the library's events switched on
+    prof_run = fresh()
+    prof_run.dec.profile_enable(True)
+    prof_run.run(timed=False)
+    prof = prof_run.dec.profile_read()
+    prof_run.dec.close()
+    dec_bytes = float(sum((c + 1) * s.kv_bytes_per_token + 2 * s.Hq * s.D * 2
+                          for ps in run.steps for c, t in zip(ps.ctx_len, ps.q_len) if t == 1))
+    pf_flops = 4.0 * s.D * s.Hq * float(sum(t * c + t * (t + 1) / 2 for ps in run.steps
+                                            for c, t in zip(ps.ctx_len, ps.q_len) if t > 1))
+
+    # end to end: every step's inputs start in pinned host memory and its output returns there
+    e2e_run = fresh(keep_host=True)
+    pinned = []
+    for ps in e2e_run.steps:
+        if ps.host is None:
+            pinned.append(None)
+            continue
+        hq, hk, hv = (torch.from_numpy(a.view(np.int16)).pin_memory() for a in ps.host)
+        pinned.append((hq, hk, hv, torch.empty_like(hq).pin_memory()))
+    e2e_run.start()
+    barrier()
+    t0 = time.perf_counter()
+    h2d = d2h = 0
+    for ps, pin in zip(e2e_run.steps, pinned):
+        e2e_run.begin_step(ps)
+        if pin is not None:
+            hq, hk, hv, ho = pin
+            e2e_run.dec.mixed_step_host(ps.slots.tolist(), ps.q_len, ps.ctx_len, hq, hk, hv, ho)
+            h2d += (hq.numel() + hk.numel() + hv.numel()) * 2
+            d2h += ho.numel() * 2
+        e2e_run.end_step(ps)
+    torch.cuda.synchronize()
+    e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
+    e2e_run.dec.close()
+    e2e = {"value": aggregate_value(tokens, world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": int(h2d / K),
+           "d2h_bytes_per_step": int(d2h / K), "steps": K, "ms_per_step": e2e_s / K * 1e3}
+    order = np.argsort(step_ms)
+    heavy = [i for i in range(K) if run.steps[i].prefill_tokens >= 4096]
+    extra = {"step_ms": {"median": float(np.median(step_ms)), "p90": float(np.percentile(step_ms, 90)),
+                         "max": float(np.max(step_ms)), "min": float(step_ms[order[0]])},
+             "sum_t_roof_over_sum_t": float(sum(t_roof) / (sum(step_ms) * 1e-3)),
+             "steps_with_prefill": int(sum(1 for ps in run.steps if ps.prefill_tokens > 0)),
+             "heavy_steps": {"count": len(heavy),
+                             "frac": float(sum(t_roof[i] for i in heavy) / (sum(step_ms[i] for i in heavy) * 1e-3)) if heavy else None}}
+    cfg = {"decode_rows": "<=%d per step" % max(ps.decode_tokens for ps in run.steps), "prefill_tokens": pf_tok,
+           "kv_tokens": None, "l2": "every step reads its own rows' K/V once; KV working set > L2 on all but the first steps"}
+    return dict(batch=None, ms_step=total_ms / K, tokens=tokens / K, prefill_tokens=pf_tok / K, decode_tokens=dec_tok / K,
+                launches=launches, clocks=clocks, prof=prof, flops=flops / K, byts=byts / K,
+                dec_bytes=dec_bytes / max(1, prof["steps"]) * 1.0, pf_flops=pf_flops / max(1, prof["steps"]) * 1.0,
+                e2e=e2e, cfg=cfg, steps=K, warmup=K, extra=extra)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    world, rank, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    r = (run_replay if args.workload == "config5" else run_static)(args, world, rank, local, barrier)
+    peaks, peak_kind = load_peaks()
+    roofline, step_roofline = rooflines(peaks, peak_kind, r["flops"], r["byts"], r["dec_bytes"], r["pf_flops"],
+                                        r["ms_step"], r["prof"])
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        leg = OracleLeg(batch)
-        stride = leg.stride_for(15.0)
-        sel = oracle_sample(batch, stride)
-        t = leg.run(sel)
-        cpu_baseline = {"value": len(sel) / t, "unit": UNIT, "cores": leg.cores, "kind": "oracle",
-                        "sample": f"every {stride}th decode row and every {stride}th prefill token "
-                                  f"({len(sel)} of {tokens} tokens), {t:.1f} s"}
-
+        cpu_baseline = cpu_baseline_leg(r["batch"] if r["batch"] is not None else make_static_batch(args.workload, 0))
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-                "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": args.workload, "description": desc, "n_q_heads": s.Hq,
-                           "n_kv_heads": s.Hkv, "head_dim": s.D, "page_size": s.P,
-                           "decode_rows": batch.decode_tokens, "prefill_tokens": batch.prefill_tokens,
-                           "kv_tokens": kv_tokens, "parallelism": f"replicas x{world}",
-                           "l2": "inputs larger than L2 (KV working set %.2f GB)" % (kv_tokens * s.kv_bytes_per_token / 1e9)},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-                "step_roofline": step_roofline, "cpu_baseline": cpu_baseline,
-                "prefill_tokens_per_s": world * batch.prefill_tokens / (ms_step * 1e-3),
-                "decode_tokens_per_s": world * batch.decode_tokens / (ms_step * 1e-3)}
+        shape = wl.LLAMA70B if args.workload == "config5" else wl.LLAMA8B
+        cfg = {"workload": args.workload, "description": WORKLOADS[args.workload][1], "n_q_heads": shape.Hq,
+               "n_kv_heads": shape.Hkv, "head_dim": shape.D, "page_size": shape.P,
+               "parallelism": f"replicas x{world}"}
+        cfg.update(r["cfg"])
+        line = {"metric": METRIC, "value": aggregate_value(r["tokens"], world, r["ms_step"] * 1e-3), "unit": UNIT,
+                "n_gpus": world, "steps": r["steps"], "warmup": r["warmup"], "ms_per_step": r["ms_step"],
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+                "data": "synthetic", "config": cfg, "clocks": r["clocks"], "e2e": r["e2e"],
+                "gpu_launches": r["launches"], "roofline": roofline, "step_roofline": step_roofline,
+                "cpu_baseline": cpu_baseline,
+                "prefill_tokens_per_s": aggregate_value(r["prefill_tokens"], world, r["ms_step"] * 1e-3),
+                "decode_tokens_per_s": aggregate_value(r["decode_tokens"], world, r["ms_step"] * 1e-3)}
+        line.update(r["extra"])
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

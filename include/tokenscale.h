@@ -176,6 +176,14 @@ typedef struct {
 } ts_step;
 
 /*
+ * ts_alloc_step: ts_alloc_pages for every row of a step in one call -- grows slot[r]'s table to
+ * ctx_len[r] + q_len[r] tokens (rows with q_len > 1 count as prefill work and may use the reserved
+ * pages). Stops at the first row that cannot be served and returns its error; rows before it
+ * keep their new pages. Only slot, q_len and ctx_len of the step are read.
+ */
+int ts_alloc_step(ts_ctx* ctx, const ts_step* step);
+
+/*
  * ts_kv_append: write the step's new K/V into the rows' pages (Sec. 2.1) and, unless
  * TS_STEP_KEEP_LEN, advance the cached lengths. q and out are ignored. Asynchronous on
  * cuda_stream (a cudaStream_t passed as void*; NULL = legacy default stream). Also the way
@@ -228,9 +236,10 @@ int ts_report_step_time(ts_ctx* ctx, double seconds);
  * clears them. Not meant for production steps (each event costs a little stream time).
  */
 typedef struct {
-  double append_ms;     /* KV append kernel                       */
-  double attention_ms;  /* attention kernel (decode splits + prefill tiles) */
-  double combine_ms;    /* split-combine kernel                   */
+  double append_ms;     /* table update + KV append kernels                  */
+  double prefill_ms;    /* prefill-chunk attention kernel                    */
+  double decode_ms;     /* split-KV decode attention kernel                  */
+  double combine_ms;    /* split-combine kernel                              */
   int64_t steps;
 } ts_profile;
 int ts_profile_enable(ts_ctx* ctx, int enable);

@@ -57,8 +57,8 @@ class ts_velocity_counters(ctypes.Structure):
 
 
 class ts_profile(ctypes.Structure):
-    _fields_ = [("append_ms", ctypes.c_double), ("attention_ms", ctypes.c_double),
-                ("combine_ms", ctypes.c_double), ("steps", ctypes.c_int64)]
+    _fields_ = [("append_ms", ctypes.c_double), ("prefill_ms", ctypes.c_double),
+                ("decode_ms", ctypes.c_double), ("combine_ms", ctypes.c_double), ("steps", ctypes.c_int64)]
 
 
 EXPORTS = ["ts_pool_bytes", "ts_workspace_bytes", "ts_create", "ts_destroy", "ts_request_add",
@@ -66,7 +66,7 @@ EXPORTS = ["ts_pool_bytes", "ts_workspace_bytes", "ts_create", "ts_destroy", "ts
            "ts_request_set_len", "ts_kv_append", "ts_mixed_step", "ts_mixed_step_host",
            "ts_velocity", "ts_report_step_time", "ts_prefill_budget", "ts_plan_step",
            "ts_last_device_status", "ts_last_cuda_error", "ts_strerror", "ts_profile_enable",
-           "ts_profile_read", "ts_decode_attention_static"]
+           "ts_profile_read", "ts_decode_attention_static", "ts_alloc_step"]
 
 _lib = None
 
@@ -98,6 +98,7 @@ def lib() -> ctypes.CDLL:
         L.ts_block_table_set.argtypes = [vp, ctypes.c_int32, _i32p, ctypes.c_int32]
         L.ts_request_free.argtypes = [vp, ctypes.c_int32]
         L.ts_request_set_len.argtypes = [vp, ctypes.c_int32, ctypes.c_int32]
+        L.ts_alloc_step.argtypes = [vp, stepp]
         L.ts_kv_append.argtypes = [vp, stepp, vp]
         L.ts_mixed_step.argtypes = [vp, stepp, vp]
         L.ts_mixed_step_host.argtypes = [vp, stepp, vp]
@@ -182,6 +183,21 @@ def make_step(slots, q_len, ctx_len, q=0, k_new=0, v_new=0, out=0, flags: int = 
     a_c = (ctypes.c_int32 * max(n, 1))(*[int(x) for x in ctx_len])
     st = ts_step(n, flags, a_slot, a_q, a_c, q or None, k_new or None, v_new or None, out or None)
     return st, (a_slot, a_q, a_c)
+
+
+def make_step_np(slots, q_len, ctx_len, q=0, k_new=0, v_new=0, out=0, flags: int = 0):
+    """Like make_step, for contiguous numpy int32 arrays: no per-element conversion.
+    Returns (step, keepalive); the arrays must stay alive while the step is used."""
+    import numpy as np
+    arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in (slots, q_len, ctx_len)]
+    ptrs = [a.ctypes.data_as(_i32p) for a in arrs]
+    st = ts_step(len(arrs[0]), flags, ptrs[0], ptrs[1], ptrs[2], q or None, k_new or None, v_new or None,
+                 out or None)
+    return st, arrs
+
+
+def ts_alloc_step(ctx, step: ts_step) -> int:
+    return lib().ts_alloc_step(ctx, ctypes.byref(step))
 
 
 def ts_kv_append(ctx, step: ts_step, cuda_stream: int = 0) -> int:

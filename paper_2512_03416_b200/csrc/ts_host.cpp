@@ -128,7 +128,7 @@ struct ts_ctx {
   std::vector<CombineItem> combines;
   std::vector<int32_t> tok0;
   std::vector<TableDelta> deltas;
-  // optional per-kernel timing: 4 events per recorded step
+  // optional per-kernel timing: 5 events per recorded step
   bool profiling = false;
   std::vector<cudaEvent_t> prof_events;
   size_t prof_used = 0;
@@ -445,15 +445,15 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
   d.n_combines = n_combines;
   cudaEvent_t* pe = nullptr;
   if (attention && c->profiling) {
-    if (c->prof_used + 4 > c->prof_events.size()) {
-      for (int i = 0; i < 4; ++i) {
+    if (c->prof_used + 5 > c->prof_events.size()) {
+      for (int i = 0; i < 5; ++i) {
         cudaEvent_t e;
         TS_CUDA(c, cudaEventCreate(&e));
         c->prof_events.push_back(e);
       }
     }
     pe = c->prof_events.data() + c->prof_used;
-    c->prof_used += 4;
+    c->prof_used += 5;
     TS_CUDA(c, cudaEventRecord(pe[0], stream));
   }
   TS_CUDA(c, ts::launch_kv_append(d, stream));
@@ -474,16 +474,17 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
       }
       ++c->cnt.kernel_launches;
     }
+    if (pe) TS_CUDA(c, cudaEventRecord(pe[2], stream));
     if (n_items > c->n_prefill_items) {
       TS_CUDA(c, ts::launch_decode(d, c->kv_map, c->n_sms, stream));
       ++c->cnt.kernel_launches;
     }
-    if (pe) TS_CUDA(c, cudaEventRecord(pe[2], stream));
+    if (pe) TS_CUDA(c, cudaEventRecord(pe[3], stream));
     if (n_combines > 0) {
       TS_CUDA(c, ts::launch_combine(d, stream));
       ++c->cnt.kernel_launches;
     }
-    if (pe) TS_CUDA(c, cudaEventRecord(pe[3], stream));
+    if (pe) TS_CUDA(c, cudaEventRecord(pe[4], stream));
     ++c->cnt.steps;
     c->cnt.prefill_tokens += (uint64_t)n_prefill;
     c->cnt.decode_tokens += (uint64_t)n_decode;
@@ -592,6 +593,17 @@ int ts_alloc_pages(ts_ctx* c, int32_t slot, int32_t total_tokens, int32_t for_pr
     c->free_pages.pop_back();
     c->page_owner[p] = slot;
     row[s.n_pages++] = p;
+  }
+  return TS_OK;
+}
+
+int ts_alloc_step(ts_ctx* c, const ts_step* st) {
+  if (!c || !st || st->n_rows < 0) return TS_ERR_INVALID;
+  if (st->n_rows > 0 && (!st->slot || !st->q_len || !st->ctx_len)) return TS_ERR_INVALID;
+  for (int r = 0; r < st->n_rows; ++r) {
+    if (st->q_len[r] < 1 || st->ctx_len[r] < 0) return TS_ERR_INVALID;
+    const int rc = ts_alloc_pages(c, st->slot[r], st->ctx_len[r] + st->q_len[r], st->q_len[r] > 1);
+    if (rc != TS_OK) return rc;
   }
   return TS_OK;
 }
@@ -729,14 +741,14 @@ int ts_profile_read(ts_ctx* c, void* cuda_stream, ts_profile* out) {
   if (c->prof_used == 0) return TS_OK;
   TS_CUDA(c, cudaSetDevice(c->cfg.device));
   TS_CUDA(c, cudaStreamSynchronize((cudaStream_t)cuda_stream));
-  for (size_t i = 0; i + 4 <= c->prof_used; i += 4) {
-    float a = 0.f, b = 0.f, d = 0.f;
-    TS_CUDA(c, cudaEventElapsedTime(&a, c->prof_events[i], c->prof_events[i + 1]));
-    TS_CUDA(c, cudaEventElapsedTime(&b, c->prof_events[i + 1], c->prof_events[i + 2]));
-    TS_CUDA(c, cudaEventElapsedTime(&d, c->prof_events[i + 2], c->prof_events[i + 3]));
-    out->append_ms += a;
-    out->attention_ms += b;
-    out->combine_ms += d;
+  for (size_t i = 0; i + 5 <= c->prof_used; i += 5) {
+    float t[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int k = 0; k < 4; ++k)
+      TS_CUDA(c, cudaEventElapsedTime(&t[k], c->prof_events[i + k], c->prof_events[i + k + 1]));
+    out->append_ms += t[0];
+    out->prefill_ms += t[1];
+    out->decode_ms += t[2];
+    out->combine_ms += t[3];
     out->steps += 1;
   }
   c->prof_used = 0;

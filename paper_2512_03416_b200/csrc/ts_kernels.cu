@@ -113,15 +113,30 @@ __global__ void combine_kernel(StepDevice s) {
   const float* ml = s.part_ml + ((size_t)c.first_partial * s.Hq + h) * 2;
   const float* pa = s.part_acc + ((size_t)c.first_partial * s.Hq + h) * s.D + d;
   const size_t ml_stride = (size_t)s.Hq * 2, pa_stride = (size_t)s.Hq * s.D;
-  float m = -CUDART_INF_F;
-#pragma unroll 8
-  for (int i = 0; i < c.n_splits; ++i) m = fmaxf(m, ml[i * ml_stride]);
-  float l = 0.f, acc = 0.f;
-#pragma unroll 8
-  for (int i = 0; i < c.n_splits; ++i) {
-    const float w = exp2f(ml[i * ml_stride] - m);
-    l += w * ml[i * ml_stride + 1];
-    acc += w * pa[i * pa_stride];
+  float m = -CUDART_INF_F, l = 0.f, acc = 0.f;
+  for (int base = 0; base < c.n_splits; base += 8) {
+    // eight splits at a time: issue every load first, then merge them into the running state
+    float mi[8], li[8], ai[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const bool on = base + j < c.n_splits;
+      mi[j] = on ? ml[(base + j) * ml_stride] : -CUDART_INF_F;
+      li[j] = on ? ml[(base + j) * ml_stride + 1] : 0.f;
+      ai[j] = on ? pa[(base + j) * pa_stride] : 0.f;
+    }
+    float mn = m;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) mn = fmaxf(mn, mi[j]);
+    const float keep = exp2f(m - mn);          // 0 on the first group (m = -inf)
+    l *= keep;
+    acc *= keep;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float w = exp2f(mi[j] - mn);       // absent split: exp2(-inf) = 0
+      l += w * li[j];
+      acc += w * ai[j];
+    }
+    m = mn;
   }
   s.out[((size_t)c.token * s.Hq + h) * s.D + d] = __bfloat16_as_ushort(__float2bfloat16_rn(acc / l));
 }

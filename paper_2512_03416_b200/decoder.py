@@ -116,6 +116,14 @@ class Decoder:
         st, _keep = self.make_step(slots, q_len, ctx_len, q, k_new, v_new, out, keep_len)
         _check(B.ts_mixed_step_host(self.ctx, st, self._stream()), "ts_mixed_step_host")
 
+    def step_np(self, slots, q_len, ctx_len, q, k_new, v_new, out, alloc: bool = True) -> None:
+        """One iteration from numpy int32 row arrays: grow the tables (ts_alloc_step), then
+        ts_mixed_step. The cheap path for per-step callers such as the trace replay."""
+        st, _keep = B.make_step_np(slots, q_len, ctx_len, _addr(q), _addr(k_new), _addr(v_new), _addr(out))
+        if alloc:
+            _check(B.ts_alloc_step(self.ctx, st), "ts_alloc_step")
+        _check(B.ts_mixed_step(self.ctx, st, self._stream()), "ts_mixed_step")
+
     def plan_step(self, slots, q_len, ctx_len):
         st, _keep = B.make_step(slots, q_len, ctx_len)
         rc, items = B.ts_plan_step(self.ctx, st)

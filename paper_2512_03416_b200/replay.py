@@ -14,7 +14,8 @@ import numpy as np
 import torch
 
 from . import workloads as wl
-from .decoder import Decoder
+from . import binding as B
+from .decoder import Decoder, TsError
 from .harness import to_dev
 
 
@@ -32,6 +33,9 @@ class PreparedStep:
     v_new: Optional[torch.Tensor] = None
     out: Optional[torch.Tensor] = None
     host: Optional[tuple] = None            # (q, k_new, v_new) bit patterns on the host, when kept
+    slots: Optional[np.ndarray] = None      # int32 slots of the rows, known once the requests are admitted
+    q_len_np: Optional[np.ndarray] = None
+    ctx_len_np: Optional[np.ndarray] = None
 
     @property
     def n_tokens(self) -> int:
@@ -67,6 +71,8 @@ class ReplayRunner:
                     live_tokens[r.req_id] = n
                 ps = PreparedStep(st.index, st.adds, st.preload, st.frees, [r[0] for r in st.rows],
                                   [r[1] for r in st.rows], [r[2] for r in st.rows])
+                ps.q_len_np = np.asarray(ps.q_len, dtype=np.int32)
+                ps.ctx_len_np = np.asarray(ps.ctx_len, dtype=np.int32)
                 n = ps.n_tokens
                 if n:
                     q, k, v = wl.replay_values(s, seed, n, self.bank)
@@ -88,27 +94,42 @@ class ReplayRunner:
                            device=device, alloc_shuffle_seed=seed, nan_fill=nan_fill,
                            decode_split_tokens=decode_split_tokens)
         self.slot_of: Dict[int, int] = {}
+        self._started = False
 
-    # -------------------------------------------------------------------------------- one step
-    def begin_step(self, ps: PreparedStep) -> None:
-        """Host bookkeeping before the step: admit requests, load warm context, grow tables."""
-        for r in ps.adds:
-            self.slot_of[r.req_id] = self.dec.request_add(r.req_id, r.prompt_len, r.output_len)
+    def start(self) -> None:
+        """Set-up that precedes the first step: admit the requests that are in flight at step 0 and
+        put their cached context into the pool (ts_kv_append). Not part of any step."""
+        if self._started:
+            return
+        self._started = True
+        ps = self.steps[0]
         for r, cached in ps.preload:
-            slot = self.slot_of[r.req_id]
+            slot = self.slot_of[r.req_id] = self.dec.request_add(r.req_id, r.prompt_len, r.output_len)
             k, v = self.warm_ctx[r.req_id]
             self.dec.alloc_pages(slot, cached, for_prefill=True)
             with torch.cuda.device(self.device):
                 self.dec.kv_append([slot], [cached], [0], to_dev(k, self.device), to_dev(v, self.device))
-        for rid, ql, ctx in zip(ps.req_ids, ps.q_len, ps.ctx_len):
-            self.dec.alloc_pages(self.slot_of[rid], ctx + ql, for_prefill=ql > 1)
+        torch.cuda.synchronize(self.device)
+
+    # -------------------------------------------------------------------------------- one step
+    def begin_step(self, ps: PreparedStep) -> None:
+        """Host bookkeeping before the step: admit new requests, grow the rows' tables."""
+        self.start()
+        for r in ps.adds:
+            if r.req_id not in self.slot_of:          # warm requests were admitted by start()
+                self.slot_of[r.req_id] = self.dec.request_add(r.req_id, r.prompt_len, r.output_len)
+        if ps.req_ids:
+            slot_of = self.slot_of
+            ps.slots = np.fromiter((slot_of[r] for r in ps.req_ids), dtype=np.int32, count=len(ps.req_ids))
+            st, keep = B.make_step_np(ps.slots, ps.q_len_np, ps.ctx_len_np)
+            rc = B.ts_alloc_step(self.dec.ctx, st)
+            if rc != B.TS_OK:
+                raise TsError(rc, "ts_alloc_step")
 
     def launch(self, ps: PreparedStep) -> None:
         if not ps.req_ids:
             return
-        with torch.cuda.device(self.device):
-            self.dec.mixed_step([self.slot_of[r] for r in ps.req_ids], ps.q_len, ps.ctx_len, ps.q, ps.k_new,
-                                ps.v_new, ps.out)
+        self.dec.step_np(ps.slots, ps.q_len_np, ps.ctx_len_np, ps.q, ps.k_new, ps.v_new, ps.out, alloc=False)
 
     def end_step(self, ps: PreparedStep) -> None:
         for rid in ps.frees:
@@ -131,6 +152,7 @@ class ReplayRunner:
     def run(self, timed: bool = True):
         """Runs every step in order; returns per-step milliseconds (CUDA events) when timed."""
         ms = []
+        self.start()
         with torch.cuda.device(self.device):
             evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
                    for _ in self.steps] if timed else None

@@ -121,14 +121,14 @@ def test_short_bursty_replay_matches_the_oracle():
     rng = np.random.default_rng(0)
     saw_prefill = saw_free = 0
     for ps in run.steps:
-        run.begin_step(ps)
+        run.begin_step(ps)                                  # the first call also loads the warm contexts
         for r, cached in ps.preload:
             k, v = run.warm_ctx[r.req_id]
             tm = _oracle_tables(run.dec, [run.slot_of[r.req_id]], width)
             oracle.kv_append(pool, s.Hkv, s.D, s.P, tm, [0], [cached], k, v)
             mirror.live[run.slot_of[r.req_id]] = cached
         if ps.req_ids:
-            slots = [run.slot_of[r] for r in ps.req_ids]
+            slots = ps.slots.tolist()
             tm = _oracle_tables(run.dec, slots, width)
             run.launch(ps)
             mirror.step(slots, ps.q_len, ps.ctx_len)
