@@ -111,12 +111,14 @@ decode_kernel(const StepDevice s, const __grid_constant__ CUtensorMap kv_map) {
   const uint32_t bars = smem_u32(merge_ml + W * G * 2);                   // [W][STAGES] mbarriers
   const uint32_t my_bars = bars + warp * STAGES * 8;
 
+  pdl_launch_dependents();
   if (tid == 0) {
     tma_prefetch_desc(&kv_map);
     for (int i = 0; i < W * STAGES; ++i) mbar_init(bars + i * 8, 1);
     mbar_init_fence();
   }
   __syncthreads();
+  pdl_wait();                  // set-up done; from here on the pool, tables and Q are read
 
   bool dead = false;           // a wait ran out: stop issuing copies, keep the control flow
   // ---------------------------------------------------------------- producer side (this warp)
@@ -348,8 +350,7 @@ cudaError_t launch_decode_t(const StepDevice& s, const CUtensorMap& map, int n_s
   if (e != cudaSuccess) return e;
   const long long units = (long long)(s.n_items - s.n_prefill_items) * s.Hkv;
   const int grid = (int)(units < n_sms ? units : n_sms);
-  decode_kernel<D, NH, STAGES><<<grid, kDecThreads, smem, stream>>>(s, map);
-  return cudaGetLastError();
+  return launch_pdl(decode_kernel<D, NH, STAGES>, dim3(grid), dim3(kDecThreads), smem, stream, s, map);
 }
 
 }  // namespace

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace ts {
 
 constexpr int kPageSize = 16;
@@ -79,5 +81,30 @@ cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream);
 // q_map views q as (head_dim, G, KV head, token), box 64 x G x 1 x 128/G.
 cudaError_t launch_prefill(const StepDevice& s, const CUtensorMap& q_map, cudaStream_t stream);
 cudaError_t launch_decode(const StepDevice& s, const CUtensorMap& kv_map, int n_sms, cudaStream_t stream);
+
+// Programmatic dependent launch: every kernel of a step is launched with the attribute that lets
+// it become resident while its predecessor in the stream is still draining. Each kernel runs its
+// set-up (shared-memory barriers, TMEM allocation, descriptor prefetch), then executes
+// griddepcontrol.wait before it touches anything an earlier kernel may have written or may still
+// be reading; launch latency and set-up thus overlap the predecessor's tail.
+template <typename... Params, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+#endif
 
 }  // namespace ts

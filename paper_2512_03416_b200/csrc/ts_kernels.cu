@@ -59,6 +59,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // ------------------------------------------------------------------------------ small kernels
 __global__ void table_update_kernel(int32_t* table, int width, int max_requests, int32_t* status,
                                     const TableDelta* deltas, int n) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const TableDelta d = deltas[i];
@@ -69,44 +71,49 @@ __global__ void table_update_kernel(int32_t* table, int width, int max_requests,
   table[(size_t)d.slot * width + d.index] = d.page;
 }
 
-// One thread per 16-byte chunk of new K or V: chunk -> (token, K|V, head, 8 elements).
+// One block per new token at a time (grid-stride over tokens); its threads copy the token's
+// 2 * Hkv * D / 8 sixteen-byte chunks of K and V. The row prefix sums sit in shared memory, so the
+// token -> row search costs no global round trips.
 __global__ void kv_append_kernel(StepDevice s) {
+  extern __shared__ int32_t row_start[];        // [n_rows + 1]
+  pdl_launch_dependents();
+  pdl_wait();
+  for (int i = threadIdx.x; i <= s.n_rows; i += blockDim.x) row_start[i] = s.row_tok0[i];
+  __syncthreads();
   const int cpr = s.D / 8;                      // chunks per (token, head) row
-  const int64_t per_tok = 2LL * s.Hkv * cpr;
-  const int64_t total = (int64_t)s.n_tokens * per_tok;
-  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-       idx += (int64_t)gridDim.x * blockDim.x) {
-    const int tok = (int)(idx / per_tok);
-    int rem = (int)(idx % per_tok);
-    const int kv = rem / (s.Hkv * cpr);
-    rem -= kv * s.Hkv * cpr;
-    const int head = rem / cpr;
-    const int ch = rem % cpr;
-    // row of this token: last r with row_tok0[r] <= tok
-    int lo = 0, hi = s.n_rows;
+  const int per_tok = 2 * s.Hkv * cpr;
+  for (int tok = blockIdx.x; tok < s.n_tokens; tok += gridDim.x) {
+    int lo = 0, hi = s.n_rows;                  // row of this token: last r with row_start[r] <= tok
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
-      if (s.row_tok0[mid] <= tok) lo = mid; else hi = mid;
+      if (row_start[mid] <= tok) lo = mid; else hi = mid;
     }
-    const int t = s.row_ctx[lo] + (tok - s.row_tok0[lo]);
+    const int t = s.row_ctx[lo] + (tok - row_start[lo]);
     const int slot = s.row_slot[lo];
     if ((unsigned)slot >= (unsigned)s.max_requests || (unsigned)(t >> 4) >= (unsigned)s.max_pages_per_req) {
-      atomicOr(s.status, TS_DEV_BAD_INDEX);
+      if (threadIdx.x == 0) atomicOr(s.status, TS_DEV_BAD_INDEX);
       continue;
     }
     const int page = s.table[(size_t)slot * s.max_pages_per_req + (t >> 4)];
     if ((unsigned)page >= (unsigned)s.n_pages) {
-      atomicOr(s.status, TS_DEV_BAD_PAGE);
+      if (threadIdx.x == 0) atomicOr(s.status, TS_DEV_BAD_PAGE);
       continue;
     }
-    const uint16_t* src = (kv ? s.v_new : s.k_new) + ((size_t)tok * s.Hkv + head) * s.D + ch * 8;
-    uint16_t* dst = s.pool + ((((size_t)page * 2 + kv) * s.Hkv + head) * kPageSize + (t & 15)) * s.D + ch * 8;
-    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+    for (int c = threadIdx.x; c < per_tok; c += blockDim.x) {
+      const int kv = c / (s.Hkv * cpr);
+      const int rem = c - kv * s.Hkv * cpr;
+      const int head = rem / cpr, ch = rem % cpr;
+      const uint16_t* src = (kv ? s.v_new : s.k_new) + ((size_t)tok * s.Hkv + head) * s.D + ch * 8;
+      uint16_t* dst = s.pool + ((((size_t)page * 2 + kv) * s.Hkv + head) * kPageSize + (t & 15)) * s.D + ch * 8;
+      *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+    }
   }
 }
 
 // Merge of the splits of one token: grid (n_combines, Hq), block D threads.
 __global__ void combine_kernel(StepDevice s) {
+  pdl_launch_dependents();
+  pdl_wait();
   const CombineItem c = s.combines[blockIdx.x];
   const int h = blockIdx.y, d = threadIdx.x;
   // the loads of different splits are independent: unrolling keeps several of them in flight
@@ -263,6 +270,8 @@ __device__ __forceinline__ void warp_tile(uint32_t sK, uint32_t sV, int key_row0
 template <int D>
 __global__ void __launch_bounds__(kThreads, 2) attention_kernel(StepDevice s) {
   extern __shared__ __align__(128) unsigned char smem[];
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int kTileBytes = kKeysPerTile * D * 2;
   const uint32_t smem_base = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -418,8 +427,7 @@ cudaError_t launch_attention_d(const StepDevice& s, cudaStream_t stream) {
   constexpr int smem = smem_pipe > smem_merge ? smem_pipe : smem_merge;
   cudaError_t e = cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  attention_kernel<D><<<dim3(s.n_items, s.Hkv), kThreads, smem, stream>>>(s);
-  return cudaGetLastError();
+  return launch_pdl(attention_kernel<D>, dim3(s.n_items, s.Hkv), dim3(kThreads), smem, stream, s);
 }
 
 }  // namespace
@@ -427,18 +435,16 @@ cudaError_t launch_attention_d(const StepDevice& s, cudaStream_t stream) {
 cudaError_t launch_table_update(int32_t* table, int max_pages_per_req, int max_requests, int32_t* status,
                                 const TableDelta* deltas, int n_deltas, cudaStream_t stream) {
   if (n_deltas <= 0) return cudaSuccess;
-  table_update_kernel<<<(n_deltas + 255) / 256, 256, 0, stream>>>(table, max_pages_per_req, max_requests, status,
-                                                                  deltas, n_deltas);
-  return cudaGetLastError();
+  return launch_pdl(table_update_kernel, dim3((n_deltas + 255) / 256), dim3(256), 0, stream, table, max_pages_per_req,
+                    max_requests, status, deltas, n_deltas);
 }
 
 cudaError_t launch_kv_append(const StepDevice& s, cudaStream_t stream) {
   if (s.n_tokens <= 0) return cudaSuccess;
-  const int64_t total = (int64_t)s.n_tokens * 2 * s.Hkv * (s.D / 8);
-  const int64_t blocks = (total + 255) / 256;
-  const int grid = (int)(blocks < 148 * 16 ? blocks : 148 * 16);
-  kv_append_kernel<<<grid, 256, 0, stream>>>(s);
-  return cudaGetLastError();
+  const int per_tok = 2 * s.Hkv * (s.D / 8);
+  const int threads = per_tok < 256 ? ((per_tok + 31) / 32) * 32 : 256;
+  const int grid = s.n_tokens < 148 * 16 ? s.n_tokens : 148 * 16;
+  return launch_pdl(kv_append_kernel, dim3(grid), dim3(threads), (s.n_rows + 1) * sizeof(int32_t), stream, s);
 }
 
 cudaError_t launch_attention(const StepDevice& s, cudaStream_t stream) {
@@ -448,8 +454,7 @@ cudaError_t launch_attention(const StepDevice& s, cudaStream_t stream) {
 
 cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream) {
   if (s.n_combines <= 0) return cudaSuccess;
-  combine_kernel<<<dim3(s.n_combines, s.Hq), s.D, 0, stream>>>(s);
-  return cudaGetLastError();
+  return launch_pdl(combine_kernel, dim3(s.n_combines, s.Hq), dim3(s.D), 0, stream, s);
 }
 
 }  // namespace ts

@@ -167,6 +167,7 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem = smem_raw + (base - smem_u32(smem_raw));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_dependents();
   const uint32_t bar0 = base + kOffBar;
   auto bar = [&](int i) { return bar0 + (uint32_t)i * 8u; };
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);  // [0] tmem base, [1] dead
@@ -199,6 +200,7 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();                  // set-up done; from here on the pool, tables and Q are read
   const uint32_t tmem = misc[0];
 
   auto give_up = [&]() {
@@ -474,8 +476,7 @@ cudaError_t launch_prefill(const StepDevice& s, const CUtensorMap& q_map, cudaSt
   if (s.n_prefill_items <= 0) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
-  prefill_kernel<<<dim3(s.Hkv, s.n_prefill_items), kPfThreads, kSmemBytes, stream>>>(s, q_map);
-  return cudaGetLastError();
+  return launch_pdl(prefill_kernel, dim3(s.Hkv, s.n_prefill_items), dim3(kPfThreads), kSmemBytes, stream, s, q_map);
 }
 
 }  // namespace ts
