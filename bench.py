@@ -31,6 +31,9 @@ from paper_2512_03416_b200 import workloads as wl  # noqa: E402
 METRIC = "prefill+decode tokens/s per B200 in mixed paged-attn step"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch on the 64 decode rows that
+# config2 and config3 share (profiles/decode_kernel_config2.md). Set to None when the kernel changes.
+DECODE_TRAFFIC_BYTES = {"config2": 7.795e8, "config3": 7.795e8}
 
 WORKLOADS = {
     "config2": (wl.config2, "decode-only batch, 8B-shaped layer (64 decode rows, ctx lognormal median 2048)"),
@@ -246,7 +249,7 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------- our arm
-def rooflines(peaks, peak_kind, flops, byts, dec_bytes, pf_flops, step_ms, prof):
+def rooflines(peaks, peak_kind, flops, byts, dec_bytes, pf_flops, step_ms, prof, traffic=None):
     steps = max(1, prof["steps"])
     dec_ms, pf_ms = prof["decode_ms"] / steps, prof["prefill_ms"] / steps
     t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
@@ -255,7 +258,7 @@ def rooflines(peaks, peak_kind, flops, byts, dec_bytes, pf_flops, step_ms, prof)
     if dec_ms >= pf_ms:
         ach = dec_bytes / (dec_ms * 1e-3) / 1e9 if dec_ms > 0 else 0.0
         roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"], "traffic": None, "kernel": "decode_kernel", "kernel_ms": dec_ms}
+                "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "kernel": "decode_kernel", "kernel_ms": dec_ms}
     else:
         ach = pf_flops / (pf_ms * 1e-3) / 1e12
         roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
@@ -447,7 +450,7 @@ def run_ours(args):
     r = (run_replay if args.workload == "config5" else run_static)(args, world, rank, local, barrier)
     peaks, peak_kind = load_peaks()
     roofline, step_roofline = rooflines(peaks, peak_kind, r["flops"], r["byts"], r["dec_bytes"], r["pf_flops"],
-                                        r["ms_step"], r["prof"])
+                                        r["ms_step"], r["prof"], DECODE_TRAFFIC_BYTES.get(args.workload))
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = cpu_baseline_leg(r["batch"] if r["batch"] is not None else make_static_batch(args.workload, 0))
