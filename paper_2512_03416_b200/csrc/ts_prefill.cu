@@ -267,9 +267,9 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
     for (int j = 0; j < nb; ++j) {
       const int st = j % stages;
       const int key0 = j * kBlockKeys;
-      int pg_next[8];
-      if (j + 1 < nb) fetch_pages(j + 1, pg_next);
       if (j >= lag) announce(j - lag, lag - 1);              // K: tile j-2 (j-1 in flight); V: tile j-1
+      int pg_next[8];
+      if (j + 1 < nb) fetch_pages(j + 1, pg_next);           // table loads fly while this tile is issued
       if (j >= stages) wait(empty + st, ((j / stages) & 1) ^ 1);
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
