@@ -25,7 +25,13 @@
 namespace ts {
 namespace {
 
-constexpr int kPfThreads = 416;                 // 8 softmax warps + 4 loader warps + MMA warp
+constexpr int kPfThreads = 512;                 // 8 softmax warps + 4 loader warps + MMA warp (+3 idle)
+// Register split (setmaxnreg works on whole warpgroups, hence the three idle warps): the block is
+// launched with 128 registers per thread; the two softmax warpgroups grow to hold a whole score
+// row, the loader and MMA warpgroups shrink. 256 * 184 + 128 * 56 + 128 * 88 = 512 * 128.
+constexpr int kRegsSoftmax = 184, kRegsLoader = 56, kRegsMma = 88;
+static_assert(256 * kRegsSoftmax + 128 * kRegsLoader + 128 * kRegsMma <= 512 * 128,
+              "register split exceeds the launch's total");
 constexpr int kLoaderThreads = 64;              // per operand (K or V)
 constexpr int kWarpLoader0 = 8, kWarpMma = 12;
 constexpr int kBlockKeys = 128;
@@ -90,7 +96,7 @@ __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint3
       "r"(a), "l"(b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(float (&v)[32], uint32_t taddr) {
+__device__ __forceinline__ void tmem_ld32(float* v, uint32_t taddr) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -105,7 +111,7 @@ __device__ __forceinline__ void tmem_ld32(float (&v)[32], uint32_t taddr) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
   const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -150,6 +156,15 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+template <int N>
+__device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(N)); }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -215,6 +230,7 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
 
   if (warp >= kWarpLoader0 && warp < kWarpLoader0 + 4) {
     // ------------------------------------------------------------------ K/V loaders
+    reg_dec<kRegsLoader>();
     // 64 threads per operand copy each 128-key tile with 16-byte cp.async straight into the
     // 128-byte-swizzled operand layout. (TMA is not used for K/V: with 16-token pages every
     // tensor copy is only 2 KB, and the copy engine's per-request cost would bound the kernel.)
@@ -293,6 +309,7 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
     for (int tile = max(0, nb - lag); tile < nb; ++tile) announce(tile, nb - 1 - tile);
   } else if (warp == kWarpMma) {
     // ------------------------------------------------------------------- MMA issuer
+    reg_dec<kRegsMma>();
     if (lane == 0) {
       constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
       // descriptors differ only in their start-address field (16-byte units in the low bits)
@@ -350,8 +367,9 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
       }
     }
     __syncwarp();
-  } else {
+  } else if (warp < 8) {
     // ------------------------------------------ softmax + epilogue: thread = query row of tile x
+    reg_inc<kRegsSoftmax>();
     const int x = warp >> 2;
     const int row = (warp & 3) * 32 + lane;
     const int nbx = x ? nb_b : nb_a;
@@ -362,35 +380,37 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
     const int lim = real ? ctx + tok + 1 : k_end_x;           // keys at positions >= lim are masked
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + x * 128 + lane_addr, tO = tmem + 256 + x * 128 + lane_addr;
+    const float scale = s.scale_log2;
     float m_ref = -CUDART_INF_F, l = 0.f;
     for (int j = 0; j < nbx; ++j) {
       wait(BAR_S_FULL + x, j & 1);
       tc_fence_after();
-      const int key0 = j * kBlockKeys;
-      const bool need_mask = key0 + kBlockKeys > lim;
-      // pass 1: row maximum of the raw scores (the scale is positive, so it commutes with max)
-      float mx = -CUDART_INF_F;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        float v[32];
-        tmem_ld32(v, tS + c * 32);
-        tmem_ld_wait();
-        if (need_mask) {
+      // the whole score row lives in registers: one trip to TMEM per block
+      float v[128];
+      tmem_ld32(&v[0], tS);
+      tmem_ld32(&v[32], tS + 32);
+      tmem_ld32(&v[64], tS + 64);
+      tmem_ld32(&v[96], tS + 96);
+      tmem_ld_wait();
+      const int nvalid = lim - j * kBlockKeys;               // keys of this block the row may see
+      if (__any_sync(0xffffffffu, nvalid < kBlockKeys)) {    // only the blocks on the diagonal
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (key0 + c * 32 + i >= lim) v[i] = -CUDART_INF_F;
-        }
-        float m0 = v[0], m1 = v[1], m2 = v[2], m3 = v[3];   // four short chains instead of one long one
-#pragma unroll
-        for (int i = 4; i < 32; i += 4) {
-          m0 = fmaxf(m0, v[i]);
-          m1 = fmaxf(m1, v[i + 1]);
-          m2 = fmaxf(m2, v[i + 2]);
-          m3 = fmaxf(m3, v[i + 3]);
-        }
-        mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
+        for (int i = 0; i < 128; ++i)
+          if (i >= nvalid) v[i] = -CUDART_INF_F;
       }
-      mx *= s.scale_log2;
+      // row maximum of the raw scores (the scale is positive, so it commutes with max)
+      float m0 = max3(v[0], v[1], v[2]), m1 = max3(v[3], v[4], v[5]);
+      float m2 = max3(v[6], v[7], v[8]), m3 = max3(v[9], v[10], v[11]);
+#pragma unroll
+      for (int i = 12; i < 124; i += 8) {
+        m0 = max3(m0, v[i], v[i + 1]);
+        m1 = max3(m1, v[i + 2], v[i + 3]);
+        m2 = max3(m2, v[i + 4], v[i + 5]);
+        m3 = max3(m3, v[i + 6], v[i + 7]);
+      }
+      m0 = max3(m0, v[124], v[125]);
+      m1 = max3(m1, v[126], v[127]);
+      const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * scale;
       // lazy rescale: move the reference maximum only when it is exceeded by 2^threshold
       const bool move = mx > m_ref + kRescaleThreshold;   // first block: m_ref = -inf, so true
       float alpha = 1.f;
@@ -412,30 +432,28 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
           tmem_st32(tO + c * 32, ov);
         }
       }
-      // pass 2: p = 2^(s*scale - m_ref), packed to bf16 over the part of S already consumed
+      // p = 2^(s*scale - m_ref), packed to bf16 over the first half of S (already in registers)
       const float neg_m = -m_ref;
-      float rs = 0.f, rs1 = 0.f;
-#pragma unroll 1
+      float rs0 = 0.f, rs1 = 0.f, rs2 = 0.f, rs3 = 0.f;
+#pragma unroll
       for (int c = 0; c < 4; ++c) {
-        float v[32];
-        tmem_ld32(v, tS + c * 32);
-        tmem_ld_wait();
         uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float p0 = ex2(fmaf(v[2 * i], s.scale_log2, neg_m));
-          float p1 = ex2(fmaf(v[2 * i + 1], s.scale_log2, neg_m));
-          if (need_mask) {
-            if (key0 + c * 32 + 2 * i >= lim) p0 = 0.f;
-            if (key0 + c * 32 + 2 * i + 1 >= lim) p1 = 0.f;
-          }
-          if (i & 1) rs1 += p0 + p1; else rs += p0 + p1;
+        for (int i = 0; i < 16; i += 2) {
+          const float p0 = ex2(fmaf(v[c * 32 + 2 * i], scale, neg_m));
+          const float p1 = ex2(fmaf(v[c * 32 + 2 * i + 1], scale, neg_m));
+          const float p2 = ex2(fmaf(v[c * 32 + 2 * i + 2], scale, neg_m));
+          const float p3 = ex2(fmaf(v[c * 32 + 2 * i + 3], scale, neg_m));
+          rs0 += p0;
+          rs1 += p1;
+          rs2 += p2;
+          rs3 += p3;
           pk[i] = pack2(p0, p1);
+          pk[i + 1] = pack2(p2, p3);
         }
-        tmem_st16(tS + c * 16, pk);       // columns [16c, 16c+16): scores there were read already
+        tmem_st16(tS + c * 16, pk);
       }
-      rs += rs1;
-      l += rs;
+      l += (rs0 + rs1) + (rs2 + rs3);
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(bar(BAR_P_FULL + x));
@@ -464,6 +482,8 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
         }
       }
     }
+  } else {
+    reg_dec<kRegsMma>();        // warps 13-15 only complete the fourth warpgroup
   }
   tc_fence_before();
   __syncthreads();
