@@ -10,7 +10,7 @@
 // while one tile's warpgroup is in its softmax, the tensor pipe works for the other tile.
 // TMEM (512 columns): S_A, S_B, O_A, O_B, 128 columns each; P overwrites the first 64 columns of
 // its S. Warp roles: warps 0-3 softmax/epilogue of tile A, warps 4-7 of tile B (thread = TMEM lane =
-// query row), warps 8-9 K loaders, warps 10-11 V loaders (16-byte cp.async through the block table
+// query row; the whole 128-score row of a block sits in the thread's registers), warps 8-9 K loaders, warps 10-11 V loaders (16-byte cp.async through the block table
 // into the swizzled operand layout), warp 12 MMA issuer and TMEM owner; the Q tiles come by TMA.
 // The O rescale is lazy: a row's reference maximum only moves when the new maximum exceeds it by
 // more than 2^8, so most blocks never touch O.
@@ -27,7 +27,7 @@ namespace {
 
 constexpr int kPfThreads = 512;                 // 8 softmax warps + 4 loader warps + MMA warp (+3 idle)
 // Register split (setmaxnreg works on whole warpgroups, hence the three idle warps): the block is
-// launched with 128 registers per thread; the two softmax warpgroups grow to hold a whole score
+// launched with 128 registers per thread; the two softmax warpgroups grow to hold their score
 // row, the loader and MMA warpgroups shrink. 256 * 184 + 128 * 56 + 128 * 88 = 512 * 128.
 constexpr int kRegsSoftmax = 184, kRegsLoader = 56, kRegsMma = 88;
 static_assert(256 * kRegsSoftmax + 128 * kRegsLoader + 128 * kRegsMma <= 512 * 128,
@@ -166,6 +166,25 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
+// Packed pairs of fp32 (sm_100 has two-wide fp32 add/fma): half the issue slots of scalar code.
+__device__ __forceinline__ uint64_t pack_f2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;\n" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;\n" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
@@ -174,6 +193,30 @@ __device__ __forceinline__ float ex2(float x) {
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// One row of a score block: p_i = 2^(v_i * scale + neg_m) for the 128 scores in v, written as bf16
+// pairs into TMEM columns [t_p, t_p + 64); returns the row sum of the unrounded p_i.
+__device__ __forceinline__ float exp_store(const float (&v)[128], float scale, float neg_m, uint32_t t_p) {
+  const uint64_t scale2 = pack_f2(scale, scale), negm2 = pack_f2(neg_m, neg_m);
+  uint64_t sum_a = pack_f2(0.f, 0.f), sum_b = sum_a;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int e = c * 32 + 2 * i;
+      float x0, x1;
+      unpack_f2(fma2(pack_f2(v[e], v[e + 1]), scale2, negm2), x0, x1);
+      const float p0 = ex2(x0), p1 = ex2(x1);
+      if (i & 1) sum_b = add2(sum_b, pack_f2(p0, p1)); else sum_a = add2(sum_a, pack_f2(p0, p1));
+      pk[i] = pack2(p0, p1);
+    }
+    tmem_st16(t_p + c * 16, pk);
+  }
+  float a0, a1;
+  unpack_f2(add2(sum_a, sum_b), a0, a1);
+  return a0 + a1;
 }
 
 __global__ void __launch_bounds__(kPfThreads, 1)
@@ -311,6 +354,14 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
     // ------------------------------------------------------------------- MMA issuer
     reg_dec<kRegsMma>();
     if (lane == 0) {
+      // the issuer keeps its own failure flag in a register: nothing on its path reads shared memory
+      bool dead = false;
+      auto wait = [&](int i, uint32_t parity) {
+        if (!mbar_wait(bar(i), parity, dead ? 2000 : kWaitCycles)) {
+          dead = true;
+          give_up();
+        }
+      };
       constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
       // descriptors differ only in their start-address field (16-byte units in the low bits)
       const uint64_t q_desc0 = smem_desc(base + kOffQ, 0, 1024);
@@ -340,7 +391,7 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
       wait(BAR_Q, 0);
       wait(BAR_K_FULL + 0, 0);
       tc_fence_after();
-      if (!misc[1]) {
+      if (!dead) {
         if (nb_a > 0) issue_qk(0, 0);
         if (nb_b > 0) issue_qk(1, 0);
         tc_commit(bar(BAR_K_EMPTY + 0));
@@ -354,14 +405,14 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
             wait(BAR_P_FULL + x, j & 1);
             if (x == 0 || j >= nb_a) wait(BAR_V_FULL + j % kVStages, (j / kVStages) & 1);
             tc_fence_after();
-            if (!misc[1]) issue_pv(x, j);
+            if (!dead) issue_pv(x, j);
           }
-          if (x == 1 && !misc[1]) tc_commit(bar(BAR_V_EMPTY + j % kVStages));   // both tiles are done with V(j)
+          if (x == 1 && !dead) tc_commit(bar(BAR_V_EMPTY + j % kVStages));   // both tiles are done with V(j)
           if (next) {
             if (x == 0 || j + 1 >= nb_a) wait(BAR_K_FULL + (j + 1) % kKStages, ((j + 1) / kKStages) & 1);
             tc_fence_after();
-            if (j + 1 < nbx && !misc[1]) issue_qk(x, j + 1);
-            if (x == 1 && !misc[1]) tc_commit(bar(BAR_K_EMPTY + (j + 1) % kKStages));
+            if (j + 1 < nbx && !dead) issue_qk(x, j + 1);
+            if (x == 1 && !dead) tc_commit(bar(BAR_K_EMPTY + (j + 1) % kKStages));
           }
         }
       }
@@ -396,7 +447,7 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
       if (__any_sync(0xffffffffu, nvalid < kBlockKeys)) {    // only the blocks on the diagonal
 #pragma unroll
         for (int i = 0; i < 128; ++i)
-          if (i >= nvalid) v[i] = -CUDART_INF_F;
+          if (i >= nvalid) v[i] = -CUDART_INF_F;             // 2^(-inf) = 0 exactly
       }
       // row maximum of the raw scores (the scale is positive, so it commutes with max)
       float m0 = max3(v[0], v[1], v[2]), m1 = max3(v[3], v[4], v[5]);
@@ -432,28 +483,8 @@ prefill_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map) {
           tmem_st32(tO + c * 32, ov);
         }
       }
-      // p = 2^(s*scale - m_ref), packed to bf16 over the first half of S (already in registers)
-      const float neg_m = -m_ref;
-      float rs0 = 0.f, rs1 = 0.f, rs2 = 0.f, rs3 = 0.f;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; i += 2) {
-          const float p0 = ex2(fmaf(v[c * 32 + 2 * i], scale, neg_m));
-          const float p1 = ex2(fmaf(v[c * 32 + 2 * i + 1], scale, neg_m));
-          const float p2 = ex2(fmaf(v[c * 32 + 2 * i + 2], scale, neg_m));
-          const float p3 = ex2(fmaf(v[c * 32 + 2 * i + 3], scale, neg_m));
-          rs0 += p0;
-          rs1 += p1;
-          rs2 += p2;
-          rs3 += p3;
-          pk[i] = pack2(p0, p1);
-          pk[i + 1] = pack2(p2, p3);
-        }
-        tmem_st16(tS + c * 16, pk);
-      }
-      l += (rs0 + rs1) + (rs2 + rs3);
+      // p = 2^(s*scale - m_ref) as bf16 over the first 64 columns of S (the scores are in registers)
+      l += exp_store(v, scale, -m_ref, tS);
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(bar(BAR_P_FULL + x));
