@@ -82,6 +82,11 @@ typedef struct {
   int32_t reserved_pages;     /* Eq. 6: pages only ts_alloc_pages(..., for_prefill=1) may take */
   int32_t decode_split_tokens;/* keys per split of a decode row; 0 = library default; rounded
                                  up to a multiple of 64                                        */
+  int32_t mixed_prefill_ctas; /* CTAs of the mixed attention kernel that only take prefill tiles
+                                 while the other CTAs stream the decode rows first (Sec. 3.4:
+                                 the decoder absorbs prefill work next to its decode batch);
+                                 0 = the library's cost model decides per step; < 0 = prefill
+                                 tiles and decode rows run as two launches, one after the other */
   float softmax_scale;        /* 0 => 1/sqrt(head_dim)                                         */
   int32_t device;             /* CUDA device ordinal that owns kv_pool and workspace           */
   uint64_t alloc_shuffle_seed;/* 0: free list hands out pages 0,1,2,...; otherwise the initial

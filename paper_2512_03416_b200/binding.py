@@ -35,7 +35,7 @@ class ts_config(ctypes.Structure):
                 ("n_pages", ctypes.c_int32), ("max_requests", ctypes.c_int32),
                 ("max_pages_per_req", ctypes.c_int32), ("chunk_size", ctypes.c_int32),
                 ("reserved_pages", ctypes.c_int32), ("decode_split_tokens", ctypes.c_int32),
-                ("softmax_scale", ctypes.c_float), ("device", ctypes.c_int32),
+                ("mixed_prefill_ctas", ctypes.c_int32), ("softmax_scale", ctypes.c_float), ("device", ctypes.c_int32),
                 ("alloc_shuffle_seed", ctypes.c_uint64),
                 ("kv_pool", ctypes.c_void_p), ("kv_pool_bytes", ctypes.c_size_t),
                 ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]

@@ -393,6 +393,7 @@ void fill_device(ts_ctx* c, const ts_step* st, int64_t n_tokens, ts::StepDevice*
   d->pool = (uint16_t*)c->cfg.kv_pool;
   d->table = (int32_t*)(ws + c->L.off_table);
   d->status = (int32_t*)(ws + c->L.off_status);
+  d->pf_queue = d->status + 1;
   d->part_acc = (float*)(ws + c->L.off_part_acc);
   d->part_ml = (float*)(ws + c->L.off_part_ml);
   d->row_slot = meta + c->L.m_row_slot;
@@ -420,6 +421,34 @@ void fill_device(ts_ctx* c, const ts_step* st, int64_t n_tokens, ts::StepDevice*
 }
 
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+// How many CTAs of the mixed kernel take prefill tiles only, the rest streaming the decode rows
+// first and joining the prefill queue afterwards. Cost model in SM-microseconds, calibrated on a
+// B200: a prefill work unit costs ~2.3 us per 128-key block pair plus ~2 us; the decode rows move
+// their K/V at a fraction of the full-chip rate that falls off as fewer SMs pull on HBM (measured:
+// 148 SMs 1.0, 120 0.955, 100 0.905, 84 0.855, 74 0.795, 64 0.69, 48 0.53, linear in between).
+int choose_prefill_ctas(const ts_ctx* c, int n_ctas, double prefill_block_pairs, double prefill_units,
+                        double decode_bytes) {
+  static const double kSm[] = {0, 48, 64, 74, 84, 100, 120, 148};
+  static const double kRate[] = {0, 0.53, 0.69, 0.795, 0.855, 0.905, 0.955, 1.0};
+  const double w_pf = prefill_block_pairs * 2.3 + prefill_units * 2.0;
+  const double t_dec_full = decode_bytes / 6.1e6;   // us at 6.1 TB/s
+  int best = 0;
+  double best_t = 1e30;
+  for (int p = 0; p < n_ctas; p += 2) {
+    const double d = (double)(n_ctas - p) * 148.0 / c->n_sms;
+    int i = 1;
+    while (i < 7 && kSm[i] < d) ++i;
+    const double rate = d >= 148.0 ? 1.0 : kRate[i - 1] + (kRate[i] - kRate[i - 1]) * (d - kSm[i - 1]) / (kSm[i] - kSm[i - 1]);
+    const double td = t_dec_full / rate;
+    const double t = std::max(td, (w_pf + (double)(n_ctas - p) * td) / n_ctas);
+    if (t < best_t - 1e-9) {
+      best_t = t;
+      best = p;
+    }
+  }
+  return best;
+}
 
 int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
   int64_t n_tokens = 0, n_prefill = 0;
@@ -461,12 +490,36 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
   if (attention) {
     if (pe) TS_CUDA(c, cudaEventRecord(pe[1], stream));
     d.n_prefill_items = c->n_prefill_items;
+    bool decode_launched = false;
     if (c->n_prefill_items > 0) {
       if (c->cfg.head_dim == 128) {
         CUtensorMap q_map;
         rc = make_q_map(c, st->q, n_tokens, &q_map);
         if (rc != TS_OK) return rc;
-        TS_CUDA(c, ts::launch_prefill(d, q_map, stream));
+        // One persistent launch: CTAs [0, p) take prefill tiles, the others run the decode
+        // splits first and then help with the tiles (decode rows ride along when G <= 8).
+        const long long pf_units = (long long)c->n_prefill_items * c->cfg.n_kv_heads;
+        const long long dec_units = (long long)(n_items - c->n_prefill_items) * c->cfg.n_kv_heads;
+        const bool fuse = dec_units > 0 && c->G <= 8 && c->cfg.mixed_prefill_ctas >= 0;
+        int n_ctas = (int)std::min<long long>(c->n_sms, pf_units + (fuse ? dec_units : 0));
+        int p = n_ctas;
+        if (fuse) {
+          if (c->cfg.mixed_prefill_ctas > 0) {
+            p = c->cfg.mixed_prefill_ctas;
+          } else {
+            double pairs = 0.0, bytes = 0.0;
+            for (int i = 0; i < c->n_prefill_items; ++i) pairs += ceil_div(c->items[i].k_end, 128);
+            for (int i = c->n_prefill_items; i < n_items; ++i)
+              bytes += (double)(c->items[i].k_end - c->items[i].k_begin);
+            bytes *= 2.0 * c->cfg.n_kv_heads * c->cfg.head_dim * 2.0;
+            p = choose_prefill_ctas(c, n_ctas, pairs * c->cfg.n_kv_heads, (double)pf_units, bytes);
+          }
+          p = (int)std::min<long long>(p, pf_units);
+          p = std::min(p, n_ctas - 1);                         // at least one CTA runs the decode splits
+          p = std::max(p, n_ctas - (int)std::min<long long>(dec_units, n_ctas));   // no CTA without a decode unit
+          decode_launched = true;
+        }
+        TS_CUDA(c, ts::launch_mixed(d, q_map, c->kv_map, n_ctas, p, stream));
       } else {
         ts::StepDevice dp = d;
         dp.n_items = c->n_prefill_items;
@@ -475,7 +528,7 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
       ++c->cnt.kernel_launches;
     }
     if (pe) TS_CUDA(c, cudaEventRecord(pe[2], stream));
-    if (n_items > c->n_prefill_items) {
+    if (n_items > c->n_prefill_items && !decode_launched) {
       TS_CUDA(c, ts::launch_decode(d, c->kv_map, c->n_sms, stream));
       ++c->cnt.kernel_launches;
     }

@@ -48,6 +48,7 @@ struct StepDevice {
   uint16_t* pool;          // caller's KV pool
   int32_t* table;          // [max_requests][max_pages_per_req]
   int32_t* status;         // device status word
+  int32_t* pf_queue;       // next prefill work unit of the step (zeroed by the append kernel)
   float* part_acc;         // [max_partials][Hq][D]
   float* part_ml;          // [max_partials][Hq][2]  (running max in log2 units, sum)
   // per step (device meta area)
@@ -77,9 +78,13 @@ cudaError_t launch_attention(const StepDevice& s, cudaStream_t stream);
 cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream);
 // Decode splits items[n_prefill_items, n_items): persistent kernel, one CTA per SM, K/V pages by TMA
 // through kv_map (5-D view of the pool: head_dim, slot, KV head, K|V, page; box 64 x 16 x 1 x 2 x 1).
-// Prefill tiles items[0, n_prefill_items), head_dim 128: tcgen05/TMEM kernel.
+// Prefill tiles items[0, n_prefill_items), head_dim 128: persistent tcgen05/TMEM kernel of n_ctas
+// CTAs. The first n_prefill_ctas CTAs work on the prefill queue only; the others first run all
+// decode splits (as launch_decode would, needs G <= 8) and then join the prefill queue. With
+// n_prefill_ctas == n_ctas the decode splits are left to launch_decode.
 // q_map views q as (head_dim, G, KV head, token), box 64 x G x 1 x 128/G.
-cudaError_t launch_prefill(const StepDevice& s, const CUtensorMap& q_map, cudaStream_t stream);
+cudaError_t launch_mixed(const StepDevice& s, const CUtensorMap& q_map, const CUtensorMap& kv_map, int n_ctas,
+                         int n_prefill_ctas, cudaStream_t stream);
 cudaError_t launch_decode(const StepDevice& s, const CUtensorMap& kv_map, int n_sms, cudaStream_t stream);
 
 // Programmatic dependent launch: every kernel of a step is launched with the attribute that lets

@@ -78,6 +78,7 @@ __global__ void kv_append_kernel(StepDevice s) {
   extern __shared__ int32_t row_start[];        // [n_rows + 1]
   pdl_launch_dependents();
   pdl_wait();
+  if (blockIdx.x == 0 && threadIdx.x == 0 && s.pf_queue) *s.pf_queue = 0;   // the step's prefill work queue
   for (int i = threadIdx.x; i <= s.n_rows; i += blockDim.x) row_start[i] = s.row_tok0[i];
   __syncthreads();
   const int cpr = s.D / 8;                      // chunks per (token, head) row
@@ -578,6 +579,7 @@ extern "C" int ts_decode_attention_static(int32_t device, int32_t n_q_heads, int
   d.pool = (uint16_t*)kv_pool;            // only read by these kernels
   d.table = (int32_t*)block_tables;       // only read
   d.status = &sc->status;
+  d.pf_queue = nullptr;
   d.part_acc = sc->part_acc;
   d.part_ml = sc->part_ml;
   d.row_slot = sc->row_slot;

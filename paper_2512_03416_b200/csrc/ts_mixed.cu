@@ -1,0 +1,705 @@
+// The attention kernel of a mixed step (sm_100a, head_dim 128): causal prefill-chunk tiles on the
+// 5th-generation tensor cores and, in the same launch, the split-KV decode units.
+//
+// One persistent CTA per SM. The first n_prefill_ctas CTAs take prefill work units (prefill work
+// item x KV head) from a global queue, heaviest first. The remaining CTAs first run their static
+// share of the decode units (dec::decode_units: TMA page copies, bound by HBM bandwidth) and then
+// join the prefill queue, so that the HBM-bound and the tensor-bound halves of a step overlap
+// instead of running back to back, and whichever CTAs finish first pick up what is left.
+//
+// A prefill work unit = two query tiles A and B of 128 packed rows each (128/G consecutive tokens
+// x the G query heads of one KV head per tile) against all keys they may see, 128 keys per block.
+// Per tile and block:
+//     S = Q K^T   (tcgen05.mma, operands in 128B-swizzled shared memory, fp32 accumulator in TMEM)
+//     online softmax by one warpgroup, one query row per thread, the score row in registers
+//     O += P V    (tcgen05.mma, P read from TMEM as bf16, V from shared memory, O accumulates in TMEM)
+// The two tiles share every K/V block (half the shared-memory fill per flop) and run out of phase:
+// while one tile's warpgroup is in its softmax, the tensor pipe works for the other tile.
+// TMEM (512 columns): S_A, S_B, O_A, O_B, 128 columns each; P overwrites the first 64 columns of
+// its S. Warp roles: warps 0-3 softmax/epilogue of tile A, warps 4-7 of tile B (thread = TMEM lane =
+// query row), warps 8-9 K loaders, warps 10-11 V loaders (16-byte cp.async through the block table
+// into the swizzled operand layout; the first K-loader thread also claims the work units), warp 12
+// MMA issuer and TMEM owner, warp 13 Q loader (TMA).
+// All barrier phases follow running block counters, so the roles flow from one work unit into the
+// next without a CTA-wide stop: the loaders run ahead into the next unit's K/V, its Q tiles land
+// as soon as the last Q K^T of the current unit has been issued, and its first Q K^T overlaps
+// the epilogue of the current unit.
+// The O rescale is lazy: a row's reference maximum only moves when the new maximum exceeds it by
+// more than 2^8, so most blocks never touch O.
+// Every wait is bounded; a wait that runs out raises TS_DEV_TIMEOUT and the CTA drains.
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include "../../include/tokenscale.h"
+#include "ts_decode_body.h"
+#include "ts_internal.h"
+#include "ts_tma.h"
+
+namespace ts {
+namespace {
+
+constexpr int kPfThreads = 512;                 // 8 softmax warps + 4 loader warps + MMA warp (+ Q-loader warp, 2 idle)
+// Register split (setmaxnreg works on whole warpgroups, hence the three idle warps): the block is
+// launched with 128 registers per thread; the two softmax warpgroups grow to hold their score
+// row, the loader and MMA warpgroups shrink. 256 * 176 + 128 * 64 + 128 * 96 = 512 * 128.
+constexpr int kRegsSoftmax = 176, kRegsLoader = 64, kRegsMma = 96;
+static_assert(256 * kRegsSoftmax + 128 * kRegsLoader + 128 * kRegsMma <= 512 * 128,
+              "register split exceeds the launch's total");
+constexpr int kLoaderThreads = 64;              // per operand (K or V)
+constexpr int kWarpLoader0 = 8, kWarpMma = 12, kWarpSched = 13;
+constexpr int kBlockKeys = 128;
+constexpr int kD = 128;
+constexpr int kTileBytes = 128 * kD * 2;        // one 128 x 128 bf16 operand tile: 32 KB
+constexpr int kHalfBytes = kTileBytes / 2;      // 64 head_dim columns of it
+constexpr int kKStages = 3, kVStages = 2;
+constexpr float kRescaleThreshold = 8.0f;       // log2 units
+
+// shared-memory map (offsets from the 1024-aligned base)
+constexpr int kOffQ = 0;                                    // Q_A, Q_B
+constexpr int kOffK = kOffQ + 2 * kTileBytes;
+constexpr int kOffV = kOffK + kKStages * kTileBytes;
+constexpr int kOffBar = kOffV + kVStages * kTileBytes;
+enum {
+  BAR_Q = 0,
+  BAR_K_FULL = 1,                         // [kKStages]
+  BAR_K_EMPTY = BAR_K_FULL + kKStages,    // [kKStages]
+  BAR_V_FULL = BAR_K_EMPTY + kKStages,    // [kVStages]
+  BAR_V_EMPTY = BAR_V_FULL + kVStages,    // [kVStages]
+  BAR_S_FULL = BAR_V_EMPTY + kVStages,    // [2] per tile
+  BAR_P_FULL = BAR_S_FULL + 2,            // [2] per tile
+  BAR_O_FULL = BAR_P_FULL + 2,            // [2] per tile
+  BAR_O_EMPTY = BAR_O_FULL + 2,           // [2] per tile: the epilogue has read O out of TMEM
+  BAR_Q_EMPTY = BAR_O_EMPTY + 2,          // the last Q K^T of a work unit has consumed the Q tiles
+  BAR_COUNT = BAR_Q_EMPTY + 1
+};
+// misc words: [0] TMEM base address, [1] failure flag, [2] work units published so far;
+// then a ring of the published units' records (8 words each)
+constexpr int kOffMisc = kOffBar + BAR_COUNT * 8;
+constexpr int kOffRing = kOffMisc + 16;
+constexpr int kSchedRing = 8;
+constexpr int kSmemBytes = kOffRing + kSchedRing * 32 + 1024;
+static_assert(kSmemBytes <= 232448, "exceeds the shared memory one CTA can opt into");
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+// ---- tcgen05 wrappers
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_dst), "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar)
+               : "memory");
+}
+// D(tmem) (+)= A(smem) * B(smem)
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d),
+      "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// D(tmem) (+)= A(tmem) * B(smem)
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(d),
+      "r"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(float* v, uint32_t taddr) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,"
+      "%27,%28,%29,%30,%31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
+  const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,"
+      "%28,%29,%30,%31,%32};\n" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+      "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
+      "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
+      "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+      "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle. `lbo`/`sbo` in bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;   // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;   // 128-byte swizzle
+  return d;
+}
+// bf16 x bf16 -> fp32, M = 128, N = 128; b_mn_major selects the layout of B.
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) |
+         ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+  // src_bytes == 0 writes 16 zero bytes and reads nothing
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+template <int N>
+__device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(N)); }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// Packed pairs of fp32 (sm_100 has two-wide fp32 add/fma): half the issue slots of scalar code.
+__device__ __forceinline__ uint64_t pack_f2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;\n" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;\n" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// One row of a score block: p_i = 2^(v_i * scale + neg_m) for the 128 scores in v, written as bf16
+// pairs into TMEM columns [t_p, t_p + 64); returns the row sum of the unrounded p_i.
+__device__ __forceinline__ float exp_store(const float (&v)[128], float scale, float neg_m, uint32_t t_p) {
+  const uint64_t scale2 = pack_f2(scale, scale), negm2 = pack_f2(neg_m, neg_m);
+  uint64_t sum_a = pack_f2(0.f, 0.f), sum_b = sum_a;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int e = c * 32 + 2 * i;
+      float x0, x1;
+      unpack_f2(fma2(pack_f2(v[e], v[e + 1]), scale2, negm2), x0, x1);
+      const float p0 = ex2(x0), p1 = ex2(x1);
+      if (i & 1) sum_b = add2(sum_b, pack_f2(p0, p1)); else sum_a = add2(sum_a, pack_f2(p0, p1));
+      pk[i] = pack2(p0, p1);
+    }
+    tmem_st16(t_p + c * 16, pk);
+  }
+  float a0, a1;
+  unpack_f2(add2(sum_a, sum_b), a0, a1);
+  return a0 + a1;
+}
+
+
+// One prefill work unit as its claimer publishes it in shared memory (8 words), and the shape
+// every role derives from it.
+struct UnitRec {
+  int32_t w;                 // work unit index, -1 = the queue is empty
+  int32_t table_slot;        // request slot: row of the block table
+  int32_t kv_head, q_begin, q_count;
+  int32_t ctx;               // tokens cached before the chunk
+  int32_t tok0;              // first token of the request row in the step's tensors
+  int32_t pad;
+};
+static_assert(sizeof(UnitRec) == 32, "UnitRec is 8 words");
+struct PfUnit {
+  int table_slot, kv_head, q_begin, ctx, tok0;
+  int cnt_a, cnt_b;          // tokens of tile A / tile B (tile B may be empty)
+  int k_end_a, k_end_b;      // one past the last key any row of the tile may see
+  int nb_a, nb_b, nb;        // key blocks per tile, and of the unit
+  int k_end;
+};
+__device__ __forceinline__ PfUnit unit_shape(const UnitRec& r, int tile_tokens) {
+  PfUnit u;
+  u.table_slot = r.table_slot;
+  u.kv_head = r.kv_head;
+  u.q_begin = r.q_begin;
+  u.ctx = r.ctx;
+  u.tok0 = r.tok0;
+  u.cnt_a = min(r.q_count, tile_tokens);
+  u.cnt_b = r.q_count - u.cnt_a;
+  u.k_end_a = u.ctx + r.q_begin + u.cnt_a;
+  u.k_end_b = u.k_end_a + u.cnt_b;
+  u.nb_a = (u.k_end_a + kBlockKeys - 1) / kBlockKeys;
+  u.nb_b = u.cnt_b > 0 ? (u.k_end_b + kBlockKeys - 1) / kBlockKeys : 0;
+  u.nb = max(u.nb_a, u.nb_b);
+  u.k_end = max(u.k_end_a, u.k_end_b);
+  return u;
+}
+
+__device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 0;\n" ::: "memory"); }
+
+__global__ void __launch_bounds__(kPfThreads, 1)
+mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
+             const __grid_constant__ CUtensorMap kv_map, const int n_prefill_ctas) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* smem = smem_raw + (base - smem_u32(smem_raw));
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_dependents();
+  const uint32_t bar0 = base + kOffBar;
+  auto bar = [&](int i) { return bar0 + (uint32_t)i * 8u; };
+  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
+  const int G = s.Hq / s.Hkv;
+  const int tile_tokens = 128 / G;
+  const int n_units = s.n_prefill_items * s.Hkv;
+  const bool decode_first = (int)blockIdx.x >= n_prefill_ctas;
+
+  auto give_up = [&]() {
+    if (misc[1] == 0) {
+      atomicOr(s.status, TS_DEV_TIMEOUT);
+      misc[1] = 1;
+    }
+  };
+  auto wait = [&](int i, uint32_t parity) {
+    if (!mbar_wait(bar(i), parity, misc[1] ? 2000 : kWaitCycles)) give_up();
+  };
+  // k-th work unit of this CTA (w = -1 after the last one), published by the K loaders' first thread
+  volatile int4* ring = reinterpret_cast<volatile int4*>(smem + kOffRing);
+  auto get_work = [&](int k, PfUnit& u) -> bool {
+    if ((int)misc[2] <= k) {
+      const long long t0 = clock64();
+      while ((int)misc[2] <= k) {
+        if (clock64() - t0 > (misc[1] ? 2000 : kWaitCycles)) {
+          give_up();
+          return false;
+        }
+      }
+    }
+    UnitRec r;
+    const int e = (k & (kSchedRing - 1)) * 2;
+    const int4 lo = make_int4(ring[e].x, ring[e].y, ring[e].z, ring[e].w);
+    const int4 hi = make_int4(ring[e + 1].x, ring[e + 1].y, ring[e + 1].z, ring[e + 1].w);
+    r.w = lo.x; r.table_slot = lo.y; r.kv_head = lo.z; r.q_begin = lo.w;
+    r.q_count = hi.x; r.ctx = hi.y; r.tok0 = hi.z;
+    if (r.w < 0) return false;
+    u = unit_shape(r, tile_tokens);
+    return true;
+  };
+  // The set-up every warp class runs between the decode phase and the prefill phase.
+  auto prefill_setup = [&]() {
+    if (tid == 0) {
+      misc[1] = 0;
+      misc[2] = 0;
+      for (int i = 0; i < BAR_COUNT; ++i) {
+        const bool softmax_arrives = (i >= BAR_P_FULL && i < BAR_P_FULL + 2) || (i >= BAR_O_EMPTY && i < BAR_O_EMPTY + 2);
+        const bool loaders_arrive = (i >= BAR_K_FULL && i < BAR_K_FULL + kKStages) ||
+                                    (i >= BAR_V_FULL && i < BAR_V_FULL + kVStages);
+        mbar_init(bar(i), softmax_arrives ? 128 : loaders_arrive ? kLoaderThreads : 1);
+      }
+      mbar_init_fence();
+    }
+    if (warp == kWarpMma) tmem_alloc(base + kOffMisc, 512);
+    tc_fence_before();
+    cta_sync();
+    tc_fence_after();
+    if (!decode_first) pdl_wait();   // set-up done; from here on the pool, tables and Q are read
+  };
+  // Decode-first CTAs: warps 0-7 run the CTA's decode units, the other warps wait for them.
+  auto decode_phase_idle = [&]() {
+    if (decode_first) {
+      pdl_wait();
+      cta_sync();
+    }
+  };
+
+  if (warp < 8) {
+    // ------------------------------------------ softmax + epilogue: thread = query row of tile x
+    reg_inc<kRegsSoftmax>();
+    if (decode_first) {
+      pdl_wait();
+      dec::decode_units<128, 1, 3>(s, &kv_map, smem, base, (int)blockIdx.x - n_prefill_ctas,
+                                   (int)gridDim.x - n_prefill_ctas);
+      fence_proxy_async();     // the prefill phase reuses this shared memory through other proxies
+      cta_sync();
+    }
+    prefill_setup();
+    const uint32_t tmem = misc[0];
+    const int x = warp >> 2;
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + x * 128 + lane_addr, tO = tmem + 256 + x * 128 + lane_addr;
+    const float scale = s.scale_log2;
+    int sx = 0;                 // blocks of this tile in earlier work units: barrier phases follow it
+    for (int k = 0;; ++k) {
+      PfUnit u;
+      if (!get_work(k, u)) break;
+      const int nbx = x ? u.nb_b : u.nb_a;
+      const int cnt = x ? u.cnt_b : u.cnt_a;
+      const int tok = u.q_begin + x * tile_tokens + row / G;   // token inside the request row
+      const bool real = row / G < cnt && row < tile_tokens * G;
+      const int lim = real ? u.ctx + tok + 1 : (x ? u.k_end_b : u.k_end_a);   // keys at positions >= lim are masked
+      const int tok0 = u.tok0;
+      float m_ref = -CUDART_INF_F, l = 0.f;
+      for (int j = 0; j < nbx; ++j) {
+        wait(BAR_S_FULL + x, (sx + j) & 1);
+        tc_fence_after();
+        // the whole score row lives in registers: one trip to TMEM per block
+        float v[128];
+        tmem_ld32(&v[0], tS);
+        tmem_ld32(&v[32], tS + 32);
+        tmem_ld32(&v[64], tS + 64);
+        tmem_ld32(&v[96], tS + 96);
+        tmem_ld_wait();
+        const int nvalid = lim - j * kBlockKeys;               // keys of this block the row may see
+        if (__any_sync(0xffffffffu, nvalid < kBlockKeys)) {    // only the blocks on the diagonal
+#pragma unroll
+          for (int i = 0; i < 128; ++i)
+            if (i >= nvalid) v[i] = -CUDART_INF_F;             // 2^(-inf) = 0 exactly
+        }
+        // row maximum of the raw scores (the scale is positive, so it commutes with max)
+        float m0 = max3(v[0], v[1], v[2]), m1 = max3(v[3], v[4], v[5]);
+        float m2 = max3(v[6], v[7], v[8]), m3 = max3(v[9], v[10], v[11]);
+#pragma unroll
+        for (int i = 12; i < 124; i += 8) {
+          m0 = max3(m0, v[i], v[i + 1]);
+          m1 = max3(m1, v[i + 2], v[i + 3]);
+          m2 = max3(m2, v[i + 4], v[i + 5]);
+          m3 = max3(m3, v[i + 6], v[i + 7]);
+        }
+        m0 = max3(m0, v[124], v[125]);
+        m1 = max3(m1, v[126], v[127]);
+        const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * scale;
+        // lazy rescale: move the reference maximum only when it is exceeded by 2^threshold
+        const bool move = mx > m_ref + kRescaleThreshold;   // first block: m_ref = -inf, so true
+        float alpha = 1.f;
+        if (move) {
+          alpha = ex2(m_ref - mx);                          // 0 on the first block
+          m_ref = mx;
+          l *= alpha;
+        }
+        if (j > 0 && __any_sync(0xffffffffu, move)) {
+          wait(BAR_O_FULL + x, (sx + j - 1) & 1);           // P V of block j-1 has landed in O
+          tc_fence_after();
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            float ov[32];
+            tmem_ld32(ov, tO + c * 32);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) ov[i] *= alpha;
+            tmem_st32(tO + c * 32, ov);
+          }
+        }
+        // p = 2^(s*scale - m_ref) as bf16 over the first 64 columns of S (the scores are in registers)
+        l += exp_store(v, scale, -m_ref, tS);
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_P_FULL + x));
+      }
+      if (nbx > 0) {
+        // epilogue: O / l -> bf16 -> global
+        wait(BAR_O_FULL + x, (sx + nbx - 1) & 1);
+        tc_fence_after();
+        const float inv = 1.f / l;
+        uint16_t* orow = s.out + ((size_t)(tok0 + tok) * s.Hq + u.kv_head * G + row % G) * kD;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float ov[32];
+          tmem_ld32(ov, tO + c * 32);
+          tmem_ld_wait();
+          if (c == 3) {
+            tc_fence_before();
+            mbar_arrive(bar(BAR_O_EMPTY + x));   // O is in registers: the next unit may overwrite it
+          }
+          if (real) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              uint4 wv;
+              wv.x = pack2(ov[8 * i] * inv, ov[8 * i + 1] * inv);
+              wv.y = pack2(ov[8 * i + 2] * inv, ov[8 * i + 3] * inv);
+              wv.z = pack2(ov[8 * i + 4] * inv, ov[8 * i + 5] * inv);
+              wv.w = pack2(ov[8 * i + 6] * inv, ov[8 * i + 7] * inv);
+              *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = wv;
+            }
+          }
+        }
+      }
+      sx += nbx;
+    }
+  } else if (warp < kWarpLoader0 + 4) {
+    // ------------------------------------------------------------------ K/V loaders
+    // 64 threads per operand copy each 128-key tile with 16-byte cp.async straight into the
+    // 128-byte-swizzled operand layout. (TMA is not used for K/V: with 16-token pages every
+    // tensor copy is only 2 KB, and the copy engine's per-request cost would bound the kernel.)
+    // K and V are two independent pipelines. A tile is announced at the start of a later
+    // iteration of its own loader, before that iteration waits for a free stage, so the
+    // announcement depends only on the copy having landed.
+    reg_dec<kRegsLoader>();
+    decode_phase_idle();
+    prefill_setup();
+    const int kv = (warp - kWarpLoader0) >> 1;               // 0: K, 1: V
+    const int t = tid - 256 - kv * kLoaderThreads;           // 0..63 inside the group
+    const int col16 = t & 15, rb = t >> 4;                   // chunk col16 of rows rb + 4 h + 8 i
+    const int stages = kv ? kVStages : kKStages;
+    const int lag = stages - 1;                              // tiles in flight besides the announced one
+    const int full = kv ? BAR_V_FULL : BAR_K_FULL, empty = kv ? BAR_V_EMPTY : BAR_K_EMPTY;
+    const uint32_t tile0 = base + (kv ? kOffV : kOffK);
+    const size_t page_stride = (size_t)2 * s.Hkv * kPageSize * kD;
+    // The first K-loader thread takes work units off the global queue, one at a time and only
+    // when the K loaders are ready for it (they run a few key blocks ahead of the tensor pipe, which
+    // hides the round trip), and publishes each to the other roles through a small ring.
+    int fetched = 0;
+    auto fetch_one = [&]() {
+      const int w = atomicAdd(s.pf_queue, 1);
+      UnitRec r = {};
+      r.w = -1;
+      if (w < n_units) {
+        const WorkItem it = s.items[w / s.Hkv];
+        r.w = w;
+        r.table_slot = s.row_slot[it.row];
+        r.kv_head = w % s.Hkv;
+        r.q_begin = it.q_begin;
+        r.q_count = it.q_count;
+        r.ctx = it.k_end - it.q_begin - it.q_count;
+        r.tok0 = s.row_tok0[it.row];
+        if ((unsigned)r.table_slot >= (unsigned)s.max_requests) {
+          atomicOr(s.status, TS_DEV_BAD_INDEX);
+          r.w = -1;
+        }
+      }
+      const int e = (fetched & (kSchedRing - 1)) * 2;
+      ring[e].x = r.w; ring[e].y = r.table_slot; ring[e].z = r.kv_head; ring[e].w = r.q_begin;
+      ring[e + 1].x = r.q_count; ring[e + 1].y = r.ctx; ring[e + 1].z = r.tok0; ring[e + 1].w = 0;
+      __threadfence_block();
+      misc[2] = (uint32_t)++fetched;
+    };
+    int g0 = 0;                                              // key blocks of earlier work units
+    for (int k = 0;; ++k) {
+      if (kv == 0 && t == 0) fetch_one();
+      PfUnit u;
+      if (!get_work(k, u)) break;
+      const int32_t* table_row = s.table + (size_t)u.table_slot * s.max_pages_per_req;
+      const size_t head_off = ((size_t)kv * s.Hkv + u.kv_head) * kPageSize * kD + col16 * 8;
+      auto fetch_pages = [&](int j, int (&pg)[8]) {
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+          const int key = j * kBlockKeys + p * kPageSize;
+          int page = -1;
+          if (key < u.k_end) {
+            page = table_row[key >> 4];
+            if ((unsigned)page >= (unsigned)s.n_pages) {
+              atomicOr(s.status, TS_DEV_BAD_PAGE);
+              page = -1;
+            }
+          }
+          pg[p] = page;
+        }
+      };
+      auto announce = [&](int tile, int pending_allowed) {   // tile = block index within the unit
+        if (pending_allowed >= 1) cp_async_wait<1>(); else cp_async_wait<0>();
+        fence_proxy_async();
+        mbar_arrive(bar(full + (g0 + tile) % stages));
+      };
+      int pg[8];
+      fetch_pages(0, pg);
+      for (int j = 0; j < u.nb; ++j) {
+        const int g = g0 + j;
+        const int st = g % stages;
+        const int key0 = j * kBlockKeys;
+        if (j >= lag) announce(j - lag, lag - 1);              // K: tile j-2 (j-1 in flight); V: tile j-1
+        int pg_next[8];
+        if (j + 1 < u.nb) fetch_pages(j + 1, pg_next);         // table loads fly while this tile is issued
+        if (g >= stages) wait(empty + st, ((g / stages) & 1) ^ 1);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int r0 = rb + 4 * h;
+          const uint32_t dst = tile0 + st * kTileBytes +
+                               (uint32_t)((col16 >> 3) * kHalfBytes + r0 * 128 + (((col16 & 7) ^ r0) << 4));
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int rowk = r0 + 8 * i;
+            const int page = pg[i >> 1];
+            const bool valid = page >= 0 && key0 + rowk < u.k_end;   // rows past the last key are zero-filled
+            const uint16_t* src = valid ? s.pool + (size_t)page * page_stride + head_off + (rowk & 15) * kD : s.pool;
+            cp_async16(dst + i * 1024, src, valid ? 16 : 0);
+          }
+        }
+        cp_async_commit();
+#pragma unroll
+        for (int p = 0; p < 8; ++p) pg[p] = pg_next[p];
+      }
+      // the last `lag` tiles (fewer when the unit is short) have not been announced yet
+      for (int tile = max(0, u.nb - lag); tile < u.nb; ++tile) announce(tile, u.nb - 1 - tile);
+      g0 += u.nb;
+    }
+  } else {
+    // ------------------------------------------------------------------- MMA issuer
+    reg_dec<kRegsMma>();          // warps 14-15 only complete the fourth warpgroup
+    decode_phase_idle();
+    prefill_setup();
+    if (warp == kWarpMma && lane == 0) {
+      const uint32_t tmem = misc[0];
+      // the issuer keeps its own failure flag in a register: nothing on its path reads shared memory
+      bool dead = false;
+      auto iwait = [&](int i, uint32_t parity) {
+        if (!mbar_wait(bar(i), parity, dead ? 2000 : kWaitCycles)) {
+          dead = true;
+          give_up();
+        }
+      };
+      constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
+      // descriptors differ only in their start-address field (16-byte units in the low bits)
+      const uint64_t q_desc0 = smem_desc(base + kOffQ, 0, 1024);
+      const uint64_t k_desc0 = smem_desc(base + kOffK, 0, 1024);
+      const uint64_t v_desc0 = smem_desc(base + kOffV, kHalfBytes, 1024);
+      auto issue_qk = [&](int x, int g) {          // S_x = Q_x K(g)^T
+        const uint64_t q_desc = q_desc0 + (uint64_t)((x * kTileBytes) >> 4);
+        const uint64_t k_desc = k_desc0 + (uint64_t)(((g % kKStages) * kTileBytes) >> 4);
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks) {
+          const uint64_t off = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+          mma_ss(tmem + x * 128, q_desc + off, k_desc + off, idesc_qk, ks > 0);
+        }
+        tc_commit(bar(BAR_S_FULL + x));
+      };
+      auto issue_pv = [&](int x, int g, bool first) {   // O_x (+)= P_x V(g)
+        const uint64_t v_desc = v_desc0 + (uint64_t)(((g % kVStages) * kTileBytes) >> 4);
+#pragma unroll
+        for (int kk = 0; kk < kBlockKeys / 16; ++kk)
+          mma_ts(tmem + 256 + x * 128, tmem + x * 128 + kk * 8, v_desc + (uint64_t)((kk * 2048) >> 4), idesc_pv,
+                 (!first || kk > 0) ? 1u : 0u);
+        tc_commit(bar(BAR_O_FULL + x));
+      };
+      int g0 = 0;                 // key blocks of earlier work units (K/V ring position)
+      int sxb[2] = {0, 0};        // blocks per tile in earlier work units (S/P/O phases)
+      int used[2] = {0, 0};       // earlier work units in which the tile had rows (O_EMPTY phases)
+      for (int k = 0;; ++k) {
+        PfUnit u;
+        if (!get_work(k, u)) break;
+        // Order: both Q K^T of block 0; then per block, for tile A then tile B:
+        // P V of block j followed at once by Q K^T of block j+1 of the same tile, so that the
+        // tile's warpgroup gets its next scores while the pipe turns to the other tile.
+        iwait(BAR_Q, k & 1);
+        iwait(BAR_K_FULL + g0 % kKStages, (g0 / kKStages) & 1);
+        tc_fence_after();
+        if (!dead) {
+          if (u.nb_a > 0) issue_qk(0, g0);
+          if (u.nb_b > 0) issue_qk(1, g0);
+          tc_commit(bar(BAR_K_EMPTY + g0 % kKStages));
+          if (u.nb == 1) tc_commit(bar(BAR_Q_EMPTY));
+        }
+        for (int j = 0; j < u.nb; ++j) {
+          const int g = g0 + j;
+          const bool next = j + 1 < u.nb;
+#pragma unroll
+          for (int x = 0; x < 2; ++x) {
+            const int nbx = x ? u.nb_b : u.nb_a;
+            if (j < nbx) {
+              iwait(BAR_P_FULL + x, (sxb[x] + j) & 1);
+              if (x == 0 || j >= u.nb_a) iwait(BAR_V_FULL + g % kVStages, (g / kVStages) & 1);
+              if (j == 0 && used[x] > 0) iwait(BAR_O_EMPTY + x, (used[x] - 1) & 1);   // the previous unit's O has been read
+              tc_fence_after();
+              if (!dead) issue_pv(x, g, j == 0);
+            }
+            if (x == 1 && !dead) tc_commit(bar(BAR_V_EMPTY + g % kVStages));   // both tiles are done with V(g)
+            if (next) {
+              if (x == 0 || j + 1 >= u.nb_a) iwait(BAR_K_FULL + (g + 1) % kKStages, ((g + 1) / kKStages) & 1);
+              tc_fence_after();
+              if (j + 1 < nbx && !dead) issue_qk(x, g + 1);
+              if (x == 1 && !dead) {
+                tc_commit(bar(BAR_K_EMPTY + (g + 1) % kKStages));
+                if (j + 2 == u.nb) tc_commit(bar(BAR_Q_EMPTY));   // that was the unit's last Q K^T
+              }
+            }
+          }
+        }
+        g0 += u.nb;
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          const int nbx = x ? u.nb_b : u.nb_a;
+          sxb[x] += nbx;
+          used[x] += nbx > 0;
+        }
+      }
+    }
+    else if (warp == kWarpSched && lane == 0) {
+      // ------------------------------------------------------------------ Q loader
+      // Brings in each work unit's Q tiles by TMA once the previous unit's last Q K^T is done.
+      tma_prefetch_desc(&q_map);
+      for (int k = 0;; ++k) {
+        PfUnit u;
+        if (!get_work(k, u)) break;
+        const int ta = u.tok0 + u.q_begin;
+        if (k > 0) wait(BAR_Q_EMPTY, (k - 1) & 1);
+        mbar_expect_tx(bar(BAR_Q), (u.cnt_b > 0 ? 2 : 1) * kTileBytes);
+        tma_load_4d(base + kOffQ, &q_map, bar(BAR_Q), 0, 0, u.kv_head, ta);
+        tma_load_4d(base + kOffQ + kHalfBytes, &q_map, bar(BAR_Q), 64, 0, u.kv_head, ta);
+        if (u.cnt_b > 0) {
+          tma_load_4d(base + kOffQ + kTileBytes, &q_map, bar(BAR_Q), 0, 0, u.kv_head, ta + tile_tokens);
+          tma_load_4d(base + kOffQ + kTileBytes + kHalfBytes, &q_map, bar(BAR_Q), 64, 0, u.kv_head, ta + tile_tokens);
+        }
+      }
+    }
+    __syncwarp();
+  }
+  tc_fence_before();
+  cta_sync();
+  if (warp == kWarpMma) tmem_dealloc(misc[0], 512);
+}
+
+}  // namespace
+
+cudaError_t launch_mixed(const StepDevice& s, const CUtensorMap& q_map, const CUtensorMap& kv_map, int n_ctas,
+                         int n_prefill_ctas, cudaStream_t stream) {
+  if (s.n_prefill_items <= 0 || n_ctas <= 0) return cudaSuccess;
+  const int G = s.Hq / s.Hkv;
+  size_t smem = kSmemBytes;
+  if (n_prefill_ctas < n_ctas) {
+    const size_t dec_smem = 1024 + dec::decode_smem_bytes<128, 3>(G);
+    if (dec_smem > smem) smem = dec_smem;
+  }
+  cudaError_t e = cudaFuncSetAttribute(mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(mixed_kernel, dim3(n_ctas), dim3(kPfThreads), smem, stream, s, q_map, kv_map, n_prefill_ctas);
+}
+
+}  // namespace ts

@@ -15,7 +15,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 def make_ctx(Hq=32, Hkv=8, D=128, n_pages=1000, max_requests=64, width=512, chunk=2112, reserved=0,
              split=0, seed=0):
-    cfg = B.ts_config(Hq, Hkv, D, 16, n_pages, max_requests, width, chunk, reserved, split, 0.0, 0, seed,
+    cfg = B.ts_config(Hq, Hkv, D, 16, n_pages, max_requests, width, chunk, reserved, split, 0, 0.0, 0, seed,
                       None, 0, None, 0)
     rc, h = B.ts_create(cfg)
     assert rc == B.TS_OK
@@ -34,11 +34,11 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_sizes_and_bad_shapes():
-    cfg = B.ts_config(32, 8, 128, 16, 100, 8, 64, 0, 0, 0, 0.0, 0, 0, None, 0, None, 0)
+    cfg = B.ts_config(32, 8, 128, 16, 100, 8, 64, 0, 0, 0, 0, 0.0, 0, 0, None, 0, None, 0)
     assert B.ts_pool_bytes(cfg) == 100 * 2 * 8 * 16 * 128 * 2
     assert B.ts_workspace_bytes(cfg) > 0
     for bad in [dict(head_dim=96), dict(page_size=32), dict(n_q_heads=30), dict(n_kv_heads=1, n_q_heads=32)]:
-        c = B.ts_config(32, 8, 128, 16, 100, 8, 64, 0, 0, 0, 0.0, 0, 0, None, 0, None, 0)
+        c = B.ts_config(32, 8, 128, 16, 100, 8, 64, 0, 0, 0, 0, 0.0, 0, 0, None, 0, None, 0)
         for k, v in bad.items():
             setattr(c, k, v)
         assert B.ts_pool_bytes(c) == 0
