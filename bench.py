@@ -31,9 +31,10 @@ from paper_2512_03416_b200 import workloads as wl  # noqa: E402
 METRIC = "prefill+decode tokens/s per B200 in mixed paged-attn step"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch on the 64 decode rows that
-# config2 and config3 share (profiles/decode_kernel_config2.md). Set to None when the kernel changes.
-DECODE_TRAFFIC_BYTES = {"config2": 7.795e8, "config3": 7.795e8}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the workload's dominant kernel, from
+# the ncu captures summarised under profiles/ (decode_kernel on config2, mixed_kernel on config3).
+# An entry is dropped (null in the output) when its kernel has changed since the capture.
+KERNEL_TRAFFIC_BYTES = {"config2": 7.795e8}
 
 WORKLOADS = {
     "config2": (wl.config2, "decode-only batch, 8B-shaped layer (64 decode rows, ctx lognormal median 2048)"),
@@ -249,24 +250,45 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------- our arm
-def rooflines(peaks, peak_kind, flops, byts, dec_bytes, pf_flops, step_ms, prof, traffic=None):
+def rooflines(peaks, peak_kind, flops, byts, dec_bytes, pf_flops, step_ms, prof, traffic=None, append_bytes=0.0):
+    """Roofline of the dominant kernel (times from the library's own CUDA events) and of the step.
+
+    Steps whose prefill tiles and decode rows ran in one launch are judged as that launch: its
+    algorithmic bytes are the step's bytes minus the append kernel's page writes, its flops the
+    step's flops, and the bound is whichever of the two takes longer at the measured peaks.
+    """
     steps = max(1, prof["steps"])
     dec_ms, pf_ms = prof["decode_ms"] / steps, prof["prefill_ms"] / steps
+    mixed_steps = prof.get("mixed_steps", 0)
+    mixed_ms = prof.get("mixed_ms", 0.0) / max(1, mixed_steps)
     t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
     t_tc = flops / (peaks["bf16_tflops"] * 1e12)
-    # the dominant kernel: decode attention (HBM) unless the prefill kernel takes longer (tensor)
-    if dec_ms >= pf_ms:
+    if mixed_steps == prof["steps"] and mixed_steps > 0:
+        k_bytes = byts - append_bytes
+        hbm_bound = k_bytes / (peaks["hbm_gbs"] * 1e9) >= t_tc
+        if hbm_bound:
+            ach = k_bytes / (mixed_ms * 1e-3) / 1e9
+            roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "kernel": "mixed_kernel", "kernel_ms": mixed_ms}
+        else:
+            ach = flops / (mixed_ms * 1e-3) / 1e12
+            roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": ach / peaks["bf16_tflops"], "traffic": None, "kernel": "mixed_kernel", "kernel_ms": mixed_ms}
+    elif dec_ms >= pf_ms:
+        # the dominant kernel: decode attention (HBM) unless the prefill kernel takes longer (tensor)
         ach = dec_bytes / (dec_ms * 1e-3) / 1e9 if dec_ms > 0 else 0.0
         roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "kernel": "decode_kernel", "kernel_ms": dec_ms}
     else:
         ach = pf_flops / (pf_ms * 1e-3) / 1e12
         roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": ach / peaks["bf16_tflops"], "traffic": None, "kernel": "prefill_kernel", "kernel_ms": pf_ms}
+                "frac": ach / peaks["bf16_tflops"], "traffic": None, "kernel": "mixed_kernel (prefill tiles only)",
+                "kernel_ms": pf_ms}
     roof.update({"peak_source": f"of {peak_kind}", "decode_ms": dec_ms, "prefill_ms": pf_ms,
+                 "mixed_ms": prof.get("mixed_ms", 0.0) / steps, "mixed_steps": mixed_steps,
                  "append_ms": prof["append_ms"] / steps, "combine_ms": prof["combine_ms"] / steps,
-                 "decode_GBps": dec_bytes / (dec_ms * 1e-3) / 1e9 if dec_ms > 0 else None,
-                 "prefill_TFLOPs": pf_flops / (pf_ms * 1e-3) / 1e12 if pf_ms > 0 else None})
+                 "decode_GBps": dec_bytes / (dec_ms * 1e-3) / 1e9 if dec_ms > 1e-3 and not mixed_steps else None,
+                 "prefill_TFLOPs": pf_flops / (pf_ms * 1e-3) / 1e12 if pf_ms > 1e-3 and not mixed_steps else None})
     t_roof = max(t_hbm, t_tc)
     step_roof = {"t_roof_us": t_roof * 1e6, "t_hbm_us": t_hbm * 1e6, "t_tensor_us": t_tc * 1e6,
                  "frac": t_roof / (step_ms * 1e-3), "flops": flops, "bytes": byts,
@@ -335,7 +357,8 @@ def run_static(args, world, rank, local, barrier):
            "l2": "inputs larger than L2 (KV working set %.2f GB)" % (kv_tokens * s.kv_bytes_per_token / 1e9)}
     return dict(batch=batch, ms_step=ms_step, tokens=tokens, prefill_tokens=batch.prefill_tokens,
                 decode_tokens=batch.decode_tokens, launches=launches, clocks=clocks, prof=prof, flops=flops,
-                byts=byts, dec_bytes=dec_bytes, pf_flops=pf_flops, e2e=e2e, cfg=cfg, steps=K, warmup=W, extra={})
+                byts=byts, dec_bytes=dec_bytes, pf_flops=pf_flops, e2e=e2e, cfg=cfg, steps=K, warmup=W, extra={},
+                append_bytes=float(batch.n_tokens * s.kv_bytes_per_token))
 
 
 def run_replay(args, world, rank, local, barrier):
@@ -450,7 +473,8 @@ def run_ours(args):
     r = (run_replay if args.workload == "config5" else run_static)(args, world, rank, local, barrier)
     peaks, peak_kind = load_peaks()
     roofline, step_roofline = rooflines(peaks, peak_kind, r["flops"], r["byts"], r["dec_bytes"], r["pf_flops"],
-                                        r["ms_step"], r["prof"], DECODE_TRAFFIC_BYTES.get(args.workload))
+                                        r["ms_step"], r["prof"], KERNEL_TRAFFIC_BYTES.get(args.workload),
+                                        r.get("append_bytes", 0.0))
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = cpu_baseline_leg(r["batch"] if r["batch"] is not None else make_static_batch(args.workload, 0))

@@ -242,10 +242,13 @@ int ts_report_step_time(ts_ctx* ctx, double seconds);
  */
 typedef struct {
   double append_ms;     /* table update + KV append kernels                  */
-  double prefill_ms;    /* prefill-chunk attention kernel                    */
-  double decode_ms;     /* split-KV decode attention kernel                  */
+  double prefill_ms;    /* attention kernel of steps whose launch held prefill tiles only */
+  double decode_ms;     /* stand-alone split-KV decode attention kernel      */
   double combine_ms;    /* split-combine kernel                              */
   int64_t steps;
+  double mixed_ms;      /* attention kernel of steps where one launch ran the prefill tiles
+                           and the decode rows together                       */
+  int64_t mixed_steps;  /* how many of `steps` those were                     */
 } ts_profile;
 int ts_profile_enable(ts_ctx* ctx, int enable);
 int ts_profile_read(ts_ctx* ctx, void* cuda_stream, ts_profile* out);

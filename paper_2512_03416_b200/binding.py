@@ -58,7 +58,8 @@ class ts_velocity_counters(ctypes.Structure):
 
 class ts_profile(ctypes.Structure):
     _fields_ = [("append_ms", ctypes.c_double), ("prefill_ms", ctypes.c_double),
-                ("decode_ms", ctypes.c_double), ("combine_ms", ctypes.c_double), ("steps", ctypes.c_int64)]
+                ("decode_ms", ctypes.c_double), ("combine_ms", ctypes.c_double), ("steps", ctypes.c_int64),
+                ("mixed_ms", ctypes.c_double), ("mixed_steps", ctypes.c_int64)]
 
 
 EXPORTS = ["ts_pool_bytes", "ts_workspace_bytes", "ts_create", "ts_destroy", "ts_request_add",

@@ -131,6 +131,7 @@ struct ts_ctx {
   // optional per-kernel timing: 5 events per recorded step
   bool profiling = false;
   std::vector<cudaEvent_t> prof_events;
+  std::vector<char> prof_mixed;     // per recorded step: did one launch run tiles and decode rows together
   size_t prof_used = 0;
 };
 
@@ -424,14 +425,14 @@ bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 // How many CTAs of the mixed kernel take prefill tiles only, the rest streaming the decode rows
 // first and joining the prefill queue afterwards. Cost model in SM-microseconds, calibrated on a
-// B200: a prefill work unit costs ~2.3 us per 128-key block pair plus ~2 us; the decode rows move
+// B200: next to streaming decode CTAs a prefill work unit costs ~3.4 us per 128-key block pair plus ~3 us; the decode rows move
 // their K/V at a fraction of the full-chip rate that falls off as fewer SMs pull on HBM (measured:
 // 148 SMs 1.0, 120 0.955, 100 0.905, 84 0.855, 74 0.795, 64 0.69, 48 0.53, linear in between).
 int choose_prefill_ctas(const ts_ctx* c, int n_ctas, double prefill_block_pairs, double prefill_units,
                         double decode_bytes) {
   static const double kSm[] = {0, 48, 64, 74, 84, 100, 120, 148};
   static const double kRate[] = {0, 0.53, 0.69, 0.795, 0.855, 0.905, 0.955, 1.0};
-  const double w_pf = prefill_block_pairs * 2.3 + prefill_units * 2.0;
+  const double w_pf = prefill_block_pairs * 3.4 + prefill_units * 3.0;
   const double t_dec_full = decode_bytes / 6.1e6;   // us at 6.1 TB/s
   int best = 0;
   double best_t = 1e30;
@@ -483,6 +484,7 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
     }
     pe = c->prof_events.data() + c->prof_used;
     c->prof_used += 5;
+    c->prof_mixed.push_back(0);
     TS_CUDA(c, cudaEventRecord(pe[0], stream));
   }
   TS_CUDA(c, ts::launch_kv_append(d, stream));
@@ -519,6 +521,7 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
           p = std::max(p, n_ctas - (int)std::min<long long>(dec_units, n_ctas));   // no CTA without a decode unit
           decode_launched = true;
         }
+        if (pe) c->prof_mixed.back() = decode_launched;
         TS_CUDA(c, ts::launch_mixed(d, q_map, c->kv_map, n_ctas, p, stream));
       } else {
         ts::StepDevice dp = d;
@@ -533,7 +536,7 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
       ++c->cnt.kernel_launches;
     }
     if (pe) TS_CUDA(c, cudaEventRecord(pe[3], stream));
-    if (n_combines > 0) {
+    if (n_combines > 0 && !decode_launched) {      // the mixed launch merges its own splits
       TS_CUDA(c, ts::launch_combine(d, stream));
       ++c->cnt.kernel_launches;
     }
@@ -799,12 +802,18 @@ int ts_profile_read(ts_ctx* c, void* cuda_stream, ts_profile* out) {
     for (int k = 0; k < 4; ++k)
       TS_CUDA(c, cudaEventElapsedTime(&t[k], c->prof_events[i + k], c->prof_events[i + k + 1]));
     out->append_ms += t[0];
-    out->prefill_ms += t[1];
+    if (c->prof_mixed[i / 5]) {
+      out->mixed_ms += t[1];
+      out->mixed_steps += 1;
+    } else {
+      out->prefill_ms += t[1];
+    }
     out->decode_ms += t[2];
     out->combine_ms += t[3];
     out->steps += 1;
   }
   c->prof_used = 0;
+  c->prof_mixed.clear();
   return TS_OK;
 }
 

@@ -48,7 +48,8 @@ struct StepDevice {
   uint16_t* pool;          // caller's KV pool
   int32_t* table;          // [max_requests][max_pages_per_req]
   int32_t* status;         // device status word
-  int32_t* pf_queue;       // next prefill work unit of the step (zeroed by the append kernel)
+  int32_t* pf_queue;       // [0] next prefill work unit of the step, [1] decode CTAs of the mixed
+                           // kernel that have finished their units (both zeroed by the append kernel)
   float* part_acc;         // [max_partials][Hq][D]
   float* part_ml;          // [max_partials][Hq][2]  (running max in log2 units, sum)
   // per step (device meta area)
@@ -81,7 +82,8 @@ cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream);
 // Prefill tiles items[0, n_prefill_items), head_dim 128: persistent tcgen05/TMEM kernel of n_ctas
 // CTAs. The first n_prefill_ctas CTAs work on the prefill queue only; the others first run all
 // decode splits (as launch_decode would, needs G <= 8) and then join the prefill queue. With
-// n_prefill_ctas == n_ctas the decode splits are left to launch_decode.
+// n_prefill_ctas == n_ctas the decode splits are left to launch_decode. When it runs the decode
+// splits it also merges them (no launch_combine needed).
 // q_map views q as (head_dim, G, KV head, token), box 64 x G x 1 x 128/G.
 cudaError_t launch_mixed(const StepDevice& s, const CUtensorMap& q_map, const CUtensorMap& kv_map, int n_ctas,
                          int n_prefill_ctas, cudaStream_t stream);
@@ -108,6 +110,41 @@ inline cudaError_t launch_pdl(void (*kernel)(Params...), dim3 grid, dim3 block, 
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 #ifdef __CUDACC__
+// Log-sum-exp merge of the splits of one (token, head) for head_dim element d: the exact merge
+//   m = max m_i,  l = sum l_i 2^(m_i - m),  O = sum acc_i 2^(m_i - m) / l
+// over the partial slots [first_partial, first_partial + n_splits). Eight splits' loads are in
+// flight at a time. Reads bypass L1 (the partials may have been written by another SM of the
+// same launch).
+__device__ __forceinline__ float merge_splits(const StepDevice& s, int first_partial, int n_splits, int h, int d) {
+  const float* ml = s.part_ml + ((size_t)first_partial * s.Hq + h) * 2;
+  const float* pa = s.part_acc + ((size_t)first_partial * s.Hq + h) * s.D + d;
+  const size_t ml_stride = (size_t)s.Hq * 2, pa_stride = (size_t)s.Hq * s.D;
+  float m = -__int_as_float(0x7f800000), l = 0.f, acc = 0.f;
+  for (int base = 0; base < n_splits; base += 8) {
+    float mi[8], li[8], ai[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const bool on = base + j < n_splits;
+      mi[j] = on ? __ldcg(ml + (base + j) * ml_stride) : -__int_as_float(0x7f800000);
+      li[j] = on ? __ldcg(ml + (base + j) * ml_stride + 1) : 0.f;
+      ai[j] = on ? __ldcg(pa + (base + j) * pa_stride) : 0.f;
+    }
+    float mn = m;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) mn = fmaxf(mn, mi[j]);
+    const float keep = exp2f(m - mn);          // 0 on the first group (m = -inf)
+    l *= keep;
+    acc *= keep;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float w = exp2f(mi[j] - mn);       // absent split: exp2(-inf) = 0
+      l += w * li[j];
+      acc += w * ai[j];
+    }
+    m = mn;
+  }
+  return acc / l;
+}
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 #endif

@@ -71,19 +71,24 @@ __global__ void table_update_kernel(int32_t* table, int width, int max_requests,
   table[(size_t)d.slot * width + d.index] = d.page;
 }
 
-// One block per new token at a time (grid-stride over tokens); its threads copy the token's
-// 2 * Hkv * D / 8 sixteen-byte chunks of K and V. The row prefix sums sit in shared memory, so the
-// token -> row search costs no global round trips.
+// One warp per new token at a time (grid-stride over tokens): its lanes copy the token's
+// 2 * Hkv * D / 8 sixteen-byte chunks of K and V, eight loads in flight per lane before the first
+// store. The row prefix sums sit in shared memory, so the token -> row search costs no global
+// round trips, and a block's warps overlap one another's table look-ups.
 __global__ void kv_append_kernel(StepDevice s) {
   extern __shared__ int32_t row_start[];        // [n_rows + 1]
   pdl_launch_dependents();
   pdl_wait();
-  if (blockIdx.x == 0 && threadIdx.x == 0 && s.pf_queue) *s.pf_queue = 0;   // the step's prefill work queue
+  if (blockIdx.x == 0 && threadIdx.x == 0 && s.pf_queue) {   // the step's work queue and decode-done count
+    s.pf_queue[0] = 0;
+    s.pf_queue[1] = 0;
+  }
   for (int i = threadIdx.x; i <= s.n_rows; i += blockDim.x) row_start[i] = s.row_tok0[i];
   __syncthreads();
+  const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cpr = s.D / 8;                      // chunks per (token, head) row
   const int per_tok = 2 * s.Hkv * cpr;
-  for (int tok = blockIdx.x; tok < s.n_tokens; tok += gridDim.x) {
+  for (int tok = blockIdx.x * warps + warp; tok < s.n_tokens; tok += gridDim.x * warps) {
     int lo = 0, hi = s.n_rows;                  // row of this token: last r with row_start[r] <= tok
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
@@ -92,21 +97,37 @@ __global__ void kv_append_kernel(StepDevice s) {
     const int t = s.row_ctx[lo] + (tok - row_start[lo]);
     const int slot = s.row_slot[lo];
     if ((unsigned)slot >= (unsigned)s.max_requests || (unsigned)(t >> 4) >= (unsigned)s.max_pages_per_req) {
-      if (threadIdx.x == 0) atomicOr(s.status, TS_DEV_BAD_INDEX);
+      if (lane == 0) atomicOr(s.status, TS_DEV_BAD_INDEX);
       continue;
     }
     const int page = s.table[(size_t)slot * s.max_pages_per_req + (t >> 4)];
     if ((unsigned)page >= (unsigned)s.n_pages) {
-      if (threadIdx.x == 0) atomicOr(s.status, TS_DEV_BAD_PAGE);
+      if (lane == 0) atomicOr(s.status, TS_DEV_BAD_PAGE);
       continue;
     }
-    for (int c = threadIdx.x; c < per_tok; c += blockDim.x) {
-      const int kv = c / (s.Hkv * cpr);
-      const int rem = c - kv * s.Hkv * cpr;
-      const int head = rem / cpr, ch = rem % cpr;
-      const uint16_t* src = (kv ? s.v_new : s.k_new) + ((size_t)tok * s.Hkv + head) * s.D + ch * 8;
-      uint16_t* dst = s.pool + ((((size_t)page * 2 + kv) * s.Hkv + head) * kPageSize + (t & 15)) * s.D + ch * 8;
-      *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+    for (int base = 0; base < per_tok; base += 256) {
+      uint4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c = base + u * 32 + lane;
+        if (c < per_tok) {
+          const int kv = c / (s.Hkv * cpr);
+          const int rem = c - kv * s.Hkv * cpr;
+          const int head = rem / cpr, ch = rem % cpr;
+          v[u] = *reinterpret_cast<const uint4*>((kv ? s.v_new : s.k_new) + ((size_t)tok * s.Hkv + head) * s.D + ch * 8);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c = base + u * 32 + lane;
+        if (c < per_tok) {
+          const int kv = c / (s.Hkv * cpr);
+          const int rem = c - kv * s.Hkv * cpr;
+          const int head = rem / cpr, ch = rem % cpr;
+          uint16_t* dst = s.pool + ((((size_t)page * 2 + kv) * s.Hkv + head) * kPageSize + (t & 15)) * s.D + ch * 8;
+          *reinterpret_cast<uint4*>(dst) = v[u];
+        }
+      }
     }
   }
 }
@@ -117,36 +138,8 @@ __global__ void combine_kernel(StepDevice s) {
   pdl_wait();
   const CombineItem c = s.combines[blockIdx.x];
   const int h = blockIdx.y, d = threadIdx.x;
-  // the loads of different splits are independent: unrolling keeps several of them in flight
-  const float* ml = s.part_ml + ((size_t)c.first_partial * s.Hq + h) * 2;
-  const float* pa = s.part_acc + ((size_t)c.first_partial * s.Hq + h) * s.D + d;
-  const size_t ml_stride = (size_t)s.Hq * 2, pa_stride = (size_t)s.Hq * s.D;
-  float m = -CUDART_INF_F, l = 0.f, acc = 0.f;
-  for (int base = 0; base < c.n_splits; base += 8) {
-    // eight splits at a time: issue every load first, then merge them into the running state
-    float mi[8], li[8], ai[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const bool on = base + j < c.n_splits;
-      mi[j] = on ? ml[(base + j) * ml_stride] : -CUDART_INF_F;
-      li[j] = on ? ml[(base + j) * ml_stride + 1] : 0.f;
-      ai[j] = on ? pa[(base + j) * pa_stride] : 0.f;
-    }
-    float mn = m;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) mn = fmaxf(mn, mi[j]);
-    const float keep = exp2f(m - mn);          // 0 on the first group (m = -inf)
-    l *= keep;
-    acc *= keep;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float w = exp2f(mi[j] - mn);       // absent split: exp2(-inf) = 0
-      l += w * li[j];
-      acc += w * ai[j];
-    }
-    m = mn;
-  }
-  s.out[((size_t)c.token * s.Hq + h) * s.D + d] = __bfloat16_as_ushort(__float2bfloat16_rn(acc / l));
+  const float o = merge_splits(s, c.first_partial, c.n_splits, h, d);
+  s.out[((size_t)c.token * s.Hq + h) * s.D + d] = __bfloat16_as_ushort(__float2bfloat16_rn(o));
 }
 
 // --------------------------------------------------------------------------- attention kernel
@@ -442,9 +435,9 @@ cudaError_t launch_table_update(int32_t* table, int max_pages_per_req, int max_r
 
 cudaError_t launch_kv_append(const StepDevice& s, cudaStream_t stream) {
   if (s.n_tokens <= 0) return cudaSuccess;
-  const int per_tok = 2 * s.Hkv * (s.D / 8);
-  const int threads = per_tok < 256 ? ((per_tok + 31) / 32) * 32 : 256;
-  const int grid = s.n_tokens < 148 * 16 ? s.n_tokens : 148 * 16;
+  const int threads = 256;                                    // eight warps = eight tokens per block at a time
+  const int blocks = (s.n_tokens + 7) / 8;
+  const int grid = blocks < 148 * 8 ? blocks : 148 * 8;
   return launch_pdl(kv_append_kernel, dim3(grid), dim3(threads), (s.n_rows + 1) * sizeof(int32_t), stream, s);
 }
 

@@ -95,24 +95,37 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar)
-               : "memory");
+// The MMA warp runs its whole loop convergently and only these three instructions are predicated
+// on one elected lane (`issue`): addresses, descriptors and loop state then stay warp-uniform,
+// which keeps them in the uniform datapath the tensor-core instructions read their operands from.
+__device__ __forceinline__ uint32_t elect_one() {
+  uint32_t pred;
+  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(pred));
+  return pred;
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t issue) {
+  asm volatile(
+      "{\n.reg .pred q;\nsetp.ne.u32 q, %1, 0;\n"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n" ::"r"(bar),
+      "r"(issue)
+      : "memory");
 }
 // D(tmem) (+)= A(smem) * B(smem)
-__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate,
+                                       uint32_t issue) {
   asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d),
-      "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      "{\n.reg .pred p, q;\nsetp.ne.u32 p, %4, 0;\nsetp.ne.u32 q, %5, 0;\n"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d),
+      "l"(a), "l"(b), "r"(idesc), "r"(accumulate), "r"(issue)
       : "memory");
 }
 // D(tmem) (+)= A(tmem) * B(smem)
-__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t accumulate,
+                                       uint32_t issue) {
   asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(d),
-      "r"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      "{\n.reg .pred p, q;\nsetp.ne.u32 p, %4, 0;\nsetp.ne.u32 q, %5, 0;\n"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(d),
+      "r"(a), "l"(b), "r"(idesc), "r"(accumulate), "r"(issue)
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(float* v, uint32_t taddr) {
@@ -358,6 +371,10 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
       pdl_wait();
       dec::decode_units<128, 1, 3>(s, &kv_map, smem, base, (int)blockIdx.x - n_prefill_ctas,
                                    (int)gridDim.x - n_prefill_ctas);
+      if (tid == 0) {          // this CTA's split partials are written: count it as done
+        __threadfence();
+        atomicAdd(s.pf_queue + 1, 1);
+      }
       fence_proxy_async();     // the prefill phase reuses this shared memory through other proxies
       cta_sync();
     }
@@ -464,6 +481,65 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
         }
       }
       sx += nbx;
+    }
+    // -------------------------------------------------------------- merge of the decode splits
+    // By now the decode CTAs are normally long done; once all of them have counted themselves,
+    // these eight warps of every CTA merge the split rows between them.
+    const int n_decode_ctas = (int)gridDim.x - n_prefill_ctas;
+    if (s.n_combines > 0 && n_decode_ctas > 0) {
+      if (tid == 0) {
+        const volatile int32_t* done = s.pf_queue + 1;
+        const long long t0 = clock64();
+        while (*done < n_decode_ctas) {
+          if (clock64() - t0 > (misc[1] ? 2000 : kWaitCycles)) {
+            give_up();
+            break;
+          }
+        }
+        __threadfence();
+      }
+      dec::block_sync();
+      // one warp per (split row, query head), dealt round-robin over all warps of the launch;
+      // a lane merges four head_dim elements
+      const int n_pairs = s.n_combines * s.Hq;
+      for (int pi = (int)blockIdx.x * 8 + warp; pi < n_pairs; pi += (int)gridDim.x * 8) {
+        const CombineItem c = s.combines[pi / s.Hq];
+        const int h = pi % s.Hq;
+        const float* ml = s.part_ml + ((size_t)c.first_partial * s.Hq + h) * 2;
+        const float* pa = s.part_acc + ((size_t)c.first_partial * s.Hq + h) * kD + lane * 4;
+        const size_t ml_stride = (size_t)s.Hq * 2, pa_stride = (size_t)s.Hq * kD;
+        float m = -CUDART_INF_F, l = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int b0 = 0; b0 < c.n_splits; b0 += 8) {
+          float mi[8], li[8];
+          float4 ai[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const bool on = b0 + j < c.n_splits;
+            mi[j] = on ? __ldcg(ml + (b0 + j) * ml_stride) : -CUDART_INF_F;
+            li[j] = on ? __ldcg(ml + (b0 + j) * ml_stride + 1) : 0.f;
+            ai[j] = on ? __ldcg(reinterpret_cast<const float4*>(pa + (b0 + j) * pa_stride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+          float mn = m;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) mn = fmaxf(mn, mi[j]);
+          const float keep = exp2f(m - mn);          // 0 on the first group (m = -inf)
+          l *= keep;
+          acc.x *= keep; acc.y *= keep; acc.z *= keep; acc.w *= keep;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float wgt = exp2f(mi[j] - mn);     // absent split: exp2(-inf) = 0
+            l += wgt * li[j];
+            acc.x += wgt * ai[j].x; acc.y += wgt * ai[j].y; acc.z += wgt * ai[j].z; acc.w += wgt * ai[j].w;
+          }
+          m = mn;
+        }
+        const float inv = 1.f / l;
+        uint2 o;
+        o.x = pack2(acc.x * inv, acc.y * inv);
+        o.y = pack2(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(s.out + ((size_t)c.token * s.Hq + h) * kD + lane * 4) = o;
+      }
     }
   } else if (warp < kWarpLoader0 + 4) {
     // ------------------------------------------------------------------ K/V loaders
@@ -576,9 +652,10 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
     reg_dec<kRegsMma>();          // warps 14-15 only complete the fourth warpgroup
     decode_phase_idle();
     prefill_setup();
-    if (warp == kWarpMma && lane == 0) {
+    if (warp == kWarpMma) {
       const uint32_t tmem = misc[0];
-      // the issuer keeps its own failure flag in a register: nothing on its path reads shared memory
+      const uint32_t issue = elect_one();
+      // the warp keeps its own failure flag in a register: nothing on its path reads shared memory
       bool dead = false;
       auto iwait = [&](int i, uint32_t parity) {
         if (!mbar_wait(bar(i), parity, dead ? 2000 : kWaitCycles)) {
@@ -597,17 +674,17 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
 #pragma unroll
         for (int ks = 0; ks < kD / 16; ++ks) {
           const uint64_t off = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
-          mma_ss(tmem + x * 128, q_desc + off, k_desc + off, idesc_qk, ks > 0);
+          mma_ss(tmem + x * 128, q_desc + off, k_desc + off, idesc_qk, ks > 0, issue);
         }
-        tc_commit(bar(BAR_S_FULL + x));
+        tc_commit(bar(BAR_S_FULL + x), issue);
       };
       auto issue_pv = [&](int x, int g, bool first) {   // O_x (+)= P_x V(g)
         const uint64_t v_desc = v_desc0 + (uint64_t)(((g % kVStages) * kTileBytes) >> 4);
 #pragma unroll
         for (int kk = 0; kk < kBlockKeys / 16; ++kk)
           mma_ts(tmem + 256 + x * 128, tmem + x * 128 + kk * 8, v_desc + (uint64_t)((kk * 2048) >> 4), idesc_pv,
-                 (!first || kk > 0) ? 1u : 0u);
-        tc_commit(bar(BAR_O_FULL + x));
+                 (!first || kk > 0) ? 1u : 0u, issue);
+        tc_commit(bar(BAR_O_FULL + x), issue);
       };
       int g0 = 0;                 // key blocks of earlier work units (K/V ring position)
       int sxb[2] = {0, 0};        // blocks per tile in earlier work units (S/P/O phases)
@@ -624,8 +701,8 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
         if (!dead) {
           if (u.nb_a > 0) issue_qk(0, g0);
           if (u.nb_b > 0) issue_qk(1, g0);
-          tc_commit(bar(BAR_K_EMPTY + g0 % kKStages));
-          if (u.nb == 1) tc_commit(bar(BAR_Q_EMPTY));
+          tc_commit(bar(BAR_K_EMPTY + g0 % kKStages), issue);
+          if (u.nb == 1) tc_commit(bar(BAR_Q_EMPTY), issue);
         }
         for (int j = 0; j < u.nb; ++j) {
           const int g = g0 + j;
@@ -640,14 +717,14 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
               tc_fence_after();
               if (!dead) issue_pv(x, g, j == 0);
             }
-            if (x == 1 && !dead) tc_commit(bar(BAR_V_EMPTY + g % kVStages));   // both tiles are done with V(g)
+            if (x == 1 && !dead) tc_commit(bar(BAR_V_EMPTY + g % kVStages), issue);   // both tiles are done with V(g)
             if (next) {
               if (x == 0 || j + 1 >= u.nb_a) iwait(BAR_K_FULL + (g + 1) % kKStages, ((g + 1) / kKStages) & 1);
               tc_fence_after();
               if (j + 1 < nbx && !dead) issue_qk(x, g + 1);
               if (x == 1 && !dead) {
-                tc_commit(bar(BAR_K_EMPTY + (g + 1) % kKStages));
-                if (j + 2 == u.nb) tc_commit(bar(BAR_Q_EMPTY));   // that was the unit's last Q K^T
+                tc_commit(bar(BAR_K_EMPTY + (g + 1) % kKStages), issue);
+                if (j + 2 == u.nb) tc_commit(bar(BAR_Q_EMPTY), issue);   // that was the unit's last Q K^T
               }
             }
           }
@@ -661,7 +738,7 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
         }
       }
     }
-    else if (warp == kWarpSched && lane == 0) {
+    if (warp == kWarpSched && lane == 0) {
       // ------------------------------------------------------------------ Q loader
       // Brings in each work unit's Q tiles by TMA once the previous unit's last Q K^T is done.
       tma_prefetch_desc(&q_map);

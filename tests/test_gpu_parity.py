@@ -97,3 +97,39 @@ def test_config4_chunked_8b(profile):
     got = run.step()
     assert_parity(got, want, profile, f"config4/{profile}")
     assert np.array_equal(run.pool(), pool_want)
+
+
+@pytest.mark.parametrize("prefill_ctas", [-1, 0, 1, 3, 100, 1000])
+def test_mixed_launch_split_invariance(prefill_ctas):
+    """The result does not depend on how the attention launch divides its CTAs between prefill
+    tiles and decode rows: two launches (-1), the cost model (0), one or three prefill CTAs (the
+    decode CTAs then take most tiles from the queue, many work units per CTA), or more prefill
+    CTAs than there are SMs (clamped)."""
+    b = wl.make_batch("mix", wl.LLAMA8B, [700, 50, 1300, 3000, 9, 0, 200], [1, 1, 1, 1, 1, 600, 130], seed=21,
+                      profile="peaked")
+    want, pool_want = oracle_step(b)
+    run = GpuRun(b, chunk_size=0, mixed_prefill_ctas=prefill_ctas)
+    got = run.step()
+    assert_parity(got, want, "peaked", f"mixed launch, prefill_ctas={prefill_ctas}")
+    assert np.array_equal(run.pool(), pool_want)
+
+
+def test_prefill_only_many_units_per_cta():
+    """A prefill-only step with more work units (tile pairs x KV heads) than SMs: every CTA of the
+    persistent kernel walks through several units, and the units differ in length."""
+    b = wl.make_batch("pf", wl.LLAMA8B, [37, 0], [1300, 75], seed=22, profile="needle")
+    want, pool_want = oracle_step(b)
+    run = GpuRun(b, chunk_size=0)
+    got = run.step()
+    assert_parity(got, want, "needle", "prefill-only, many units")
+    assert np.array_equal(run.pool(), pool_want)
+
+
+def test_mixed_70b_shape_group8():
+    """Eight query heads per KV head (the 70B-shaped layer): 16-token query tiles, decode rows in the same launch."""
+    b = wl.make_batch("m70", wl.LLAMA70B, [900, 17, 2500, 0], [1, 1, 1, 200], seed=23, profile="peaked")
+    want, pool_want = oracle_step(b)
+    run = GpuRun(b, chunk_size=0)
+    got = run.step()
+    assert_parity(got, want, "peaked", "70B-shaped mixed step")
+    assert np.array_equal(run.pool(), pool_want)
