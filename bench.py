@@ -250,45 +250,47 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------- our arm
-def rooflines(peaks, peak_kind, flops, byts, dec_bytes, pf_flops, step_ms, prof, traffic=None, append_bytes=0.0):
+def rooflines(peaks, peak_kind, flops, byts, step_ms, prof, parts, traffic=None):
     """Roofline of the dominant kernel (times from the library's own CUDA events) and of the step.
 
-    Steps whose prefill tiles and decode rows ran in one launch are judged as that launch: its
-    algorithmic bytes are the step's bytes minus the append kernel's page writes, its flops the
-    step's flops, and the bound is whichever of the two takes longer at the measured peaks.
+    `parts` holds algorithmic work per recorded step, averaged over all recorded steps:
+    dec_bytes of the steps whose decode rows ran in decode_kernel, pf_flops of the steps whose launch
+    held prefill tiles only, and mixed_bytes / mixed_flops of the steps where one launch ran tiles
+    and decode rows together (that launch does everything but the append kernel's page writes).
+    The dominant kernel is the one with the largest total time; achieved = its algorithmic work
+    over its own time.
     """
     steps = max(1, prof["steps"])
-    dec_ms, pf_ms = prof["decode_ms"] / steps, prof["prefill_ms"] / steps
-    mixed_steps = prof.get("mixed_steps", 0)
-    mixed_ms = prof.get("mixed_ms", 0.0) / max(1, mixed_steps)
+    dec_ms, pf_ms, mixed_ms = prof["decode_ms"] / steps, prof["prefill_ms"] / steps, prof.get("mixed_ms", 0.0) / steps
     t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
     t_tc = flops / (peaks["bf16_tflops"] * 1e12)
-    if mixed_steps == prof["steps"] and mixed_steps > 0:
-        k_bytes = byts - append_bytes
-        hbm_bound = k_bytes / (peaks["hbm_gbs"] * 1e9) >= t_tc
-        if hbm_bound:
-            ach = k_bytes / (mixed_ms * 1e-3) / 1e9
-            roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "kernel": "mixed_kernel", "kernel_ms": mixed_ms}
+
+    def hbm(kernel, nbytes, ms, tr=None):
+        ach = nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+        return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"], "traffic": tr, "kernel": kernel, "kernel_ms": ms}
+
+    def tensor(kernel, nflops, ms):
+        ach = nflops / (ms * 1e-3) / 1e12 if ms > 0 else 0.0
+        return {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops"], "traffic": None, "kernel": kernel, "kernel_ms": ms}
+
+    if mixed_ms >= dec_ms and mixed_ms >= pf_ms and mixed_ms > 0:
+        if parts["mixed_bytes"] / (peaks["hbm_gbs"] * 1e9) >= parts["mixed_flops"] / (peaks["bf16_tflops"] * 1e12):
+            roof = hbm("mixed_kernel", parts["mixed_bytes"], mixed_ms, traffic)
         else:
-            ach = flops / (mixed_ms * 1e-3) / 1e12
-            roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": ach / peaks["bf16_tflops"], "traffic": None, "kernel": "mixed_kernel", "kernel_ms": mixed_ms}
+            roof = tensor("mixed_kernel", parts["mixed_flops"], mixed_ms)
     elif dec_ms >= pf_ms:
-        # the dominant kernel: decode attention (HBM) unless the prefill kernel takes longer (tensor)
-        ach = dec_bytes / (dec_ms * 1e-3) / 1e9 if dec_ms > 0 else 0.0
-        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "kernel": "decode_kernel", "kernel_ms": dec_ms}
+        roof = hbm("decode_kernel", parts["dec_bytes"], dec_ms, traffic)
     else:
-        ach = pf_flops / (pf_ms * 1e-3) / 1e12
-        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": ach / peaks["bf16_tflops"], "traffic": None, "kernel": "mixed_kernel (prefill tiles only)",
-                "kernel_ms": pf_ms}
-    roof.update({"peak_source": f"of {peak_kind}", "decode_ms": dec_ms, "prefill_ms": pf_ms,
-                 "mixed_ms": prof.get("mixed_ms", 0.0) / steps, "mixed_steps": mixed_steps,
+        roof = tensor("mixed_kernel (prefill tiles only)", parts["pf_flops"], pf_ms)
+    roof.update({"peak_source": f"of {peak_kind}", "decode_ms": dec_ms, "prefill_ms": pf_ms, "mixed_ms": mixed_ms,
+                 "mixed_steps": prof.get("mixed_steps", 0), "recorded_steps": prof["steps"],
                  "append_ms": prof["append_ms"] / steps, "combine_ms": prof["combine_ms"] / steps,
-                 "decode_GBps": dec_bytes / (dec_ms * 1e-3) / 1e9 if dec_ms > 1e-3 and not mixed_steps else None,
-                 "prefill_TFLOPs": pf_flops / (pf_ms * 1e-3) / 1e12 if pf_ms > 1e-3 and not mixed_steps else None})
+                 "decode_GBps": parts["dec_bytes"] / (dec_ms * 1e-3) / 1e9 if dec_ms > 1e-3 else None,
+                 "prefill_TFLOPs": parts["pf_flops"] / (pf_ms * 1e-3) / 1e12 if pf_ms > 1e-3 else None,
+                 "mixed_GBps": parts["mixed_bytes"] / (mixed_ms * 1e-3) / 1e9 if mixed_ms > 1e-3 else None,
+                 "mixed_TFLOPs": parts["mixed_flops"] / (mixed_ms * 1e-3) / 1e12 if mixed_ms > 1e-3 else None})
     t_roof = max(t_hbm, t_tc)
     step_roof = {"t_roof_us": t_roof * 1e6, "t_hbm_us": t_hbm * 1e6, "t_tensor_us": t_tc * 1e6,
                  "frac": t_roof / (step_ms * 1e-3), "flops": flops, "bytes": byts,
@@ -333,6 +335,10 @@ def run_static(args, world, rank, local, barrier):
     dec_bytes = float(((batch.ctx_len[dec] + 1) * s.kv_bytes_per_token).sum() + 2 * dec.sum() * s.Hq * s.D * 2)
     pf_flops = 4.0 * s.D * s.Hq * float(sum(t * c + t * (t + 1) / 2 for c, t in
                                             zip(batch.ctx_len[~dec].tolist(), batch.q_len[~dec].tolist())))
+    mixed = prof.get("mixed_steps", 0) > 0          # one launch ran the tiles and the decode rows together
+    parts = {"dec_bytes": 0.0 if mixed else dec_bytes, "pf_flops": 0.0 if mixed else pf_flops,
+             "mixed_bytes": byts - batch.n_tokens * s.kv_bytes_per_token if mixed else 0.0,
+             "mixed_flops": flops if mixed else 0.0}
 
     # end to end: host buffers in, host buffer out, through ts_mixed_step_host
     Ke = min(K, 300)
@@ -357,8 +363,7 @@ def run_static(args, world, rank, local, barrier):
            "l2": "inputs larger than L2 (KV working set %.2f GB)" % (kv_tokens * s.kv_bytes_per_token / 1e9)}
     return dict(batch=batch, ms_step=ms_step, tokens=tokens, prefill_tokens=batch.prefill_tokens,
                 decode_tokens=batch.decode_tokens, launches=launches, clocks=clocks, prof=prof, flops=flops,
-                byts=byts, dec_bytes=dec_bytes, pf_flops=pf_flops, e2e=e2e, cfg=cfg, steps=K, warmup=W, extra={},
-                append_bytes=float(batch.n_tokens * s.kv_bytes_per_token))
+                byts=byts, parts=parts, e2e=e2e, cfg=cfg, steps=K, warmup=W, extra={})
 
 
 def run_replay(args, world, rank, local, barrier):
@@ -407,10 +412,22 @@ def run_replay(args, world, rank, local, barrier):
     prof_run.run(timed=False)
     prof = prof_run.dec.profile_read()
     prof_run.dec.close()
-    dec_bytes = float(sum((c + 1) * s.kv_bytes_per_token + 2 * s.Hq * s.D * 2
-                          for ps in run.steps for c, t in zip(ps.ctx_len, ps.q_len) if t == 1))
-    pf_flops = 4.0 * s.D * s.Hq * float(sum(t * c + t * (t + 1) / 2 for ps in run.steps
-                                            for c, t in zip(ps.ctx_len, ps.q_len) if t > 1))
+    # algorithmic work per kind of launch: a step with prefill tokens and decode rows runs both in one
+    # launch (G <= 8 here); a step without prefill tokens runs decode_kernel
+    dec_bytes = pf_flops = mixed_bytes = mixed_flops = 0.0
+    for ps, w in zip(run.steps, work):
+        n_dec = sum(1 for t in ps.q_len if t == 1)
+        n_new = int(sum(ps.q_len))
+        if ps.prefill_tokens > 0 and n_dec > 0:
+            mixed_bytes += w[1] - n_new * s.kv_bytes_per_token
+            mixed_flops += w[0]
+        elif ps.prefill_tokens > 0:
+            pf_flops += w[0]
+        else:
+            dec_bytes += float(sum((c + 1) * s.kv_bytes_per_token + 2 * s.Hq * s.D * 2 for c in ps.ctx_len))
+    n_rec = max(1, prof["steps"])
+    parts = {"dec_bytes": dec_bytes / n_rec, "pf_flops": pf_flops / n_rec, "mixed_bytes": mixed_bytes / n_rec,
+             "mixed_flops": mixed_flops / n_rec}
 
     # end to end: every step's inputs start in pinned host memory and its output returns there
     e2e_run = fresh(keep_host=True)
@@ -450,8 +467,7 @@ def run_replay(args, world, rank, local, barrier):
            "kv_tokens": None, "l2": "every step reads its own rows' K/V once; KV working set > L2 on all but the first steps"}
     return dict(batch=None, ms_step=total_ms / K, tokens=tokens / K, prefill_tokens=pf_tok / K, decode_tokens=dec_tok / K,
                 launches=launches, clocks=clocks, prof=prof, flops=flops / K, byts=byts / K,
-                dec_bytes=dec_bytes / max(1, prof["steps"]) * 1.0, pf_flops=pf_flops / max(1, prof["steps"]) * 1.0,
-                e2e=e2e, cfg=cfg, steps=K, warmup=K, extra=extra)
+                parts=parts, e2e=e2e, cfg=cfg, steps=K, warmup=K, extra=extra)
 
 
 def run_ours(args):
@@ -472,9 +488,8 @@ def run_ours(args):
 
     r = (run_replay if args.workload == "config5" else run_static)(args, world, rank, local, barrier)
     peaks, peak_kind = load_peaks()
-    roofline, step_roofline = rooflines(peaks, peak_kind, r["flops"], r["byts"], r["dec_bytes"], r["pf_flops"],
-                                        r["ms_step"], r["prof"], KERNEL_TRAFFIC_BYTES.get(args.workload),
-                                        r.get("append_bytes", 0.0))
+    roofline, step_roofline = rooflines(peaks, peak_kind, r["flops"], r["byts"], r["ms_step"], r["prof"], r["parts"],
+                                        KERNEL_TRAFFIC_BYTES.get(args.workload))
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = cpu_baseline_leg(r["batch"] if r["batch"] is not None else make_static_batch(args.workload, 0))
