@@ -425,13 +425,22 @@ bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 // How many CTAs of the mixed kernel take prefill tiles only, the rest streaming the decode rows
 // first and joining the prefill queue afterwards. Cost model in SM-microseconds, calibrated on a
-// B200: next to streaming decode CTAs a prefill work unit costs ~3.4 us per 128-key block pair plus ~3 us; the decode rows move
-// their K/V at a fraction of the full-chip rate that falls off as fewer SMs pull on HBM (measured:
-// 148 SMs 1.0, 120 0.955, 100 0.905, 84 0.855, 74 0.795, 64 0.69, 48 0.53, linear in between).
+// B200: next to streaming decode CTAs a prefill work unit costs ~3.4 us per 128-key block pair
+// plus ~3 us; the decode rows move their K/V at a fraction of the full-chip rate that falls off as
+// fewer SMs pull on HBM, faster with eight query heads per KV head (twice the arithmetic per page)
+// than with four. Measured (SMs -> fraction, linear in between):
+//   G <= 4:  48 0.53,  64 0.69, 74 0.795, 84 0.855, 100 0.905, 120 0.955, 148 1
+//   G >  4:  48 0.475, 64 0.62, 74 0.715, 84 0.78,  100 0.85,  116 0.92, 132 0.95, 148 1
 int choose_prefill_ctas(const ts_ctx* c, int n_ctas, double prefill_block_pairs, double prefill_units,
                         double decode_bytes) {
-  static const double kSm[] = {0, 48, 64, 74, 84, 100, 120, 148};
-  static const double kRate[] = {0, 0.53, 0.69, 0.795, 0.855, 0.905, 0.955, 1.0};
+  static const double kSm4[] = {0, 48, 64, 74, 84, 100, 120, 148};
+  static const double kRate4[] = {0, 0.53, 0.69, 0.795, 0.855, 0.905, 0.955, 1.0};
+  static const double kSm8[] = {0, 48, 64, 74, 84, 100, 116, 132, 148};
+  static const double kRate8[] = {0, 0.475, 0.62, 0.715, 0.78, 0.85, 0.92, 0.95, 1.0};
+  const bool wide = c->G > 4;
+  const double* kSm = wide ? kSm8 : kSm4;
+  const double* kRate = wide ? kRate8 : kRate4;
+  const int last = wide ? 8 : 7;
   const double w_pf = prefill_block_pairs * 3.4 + prefill_units * 3.0;
   const double t_dec_full = decode_bytes / 6.1e6;   // us at 6.1 TB/s
   int best = 0;
@@ -439,7 +448,7 @@ int choose_prefill_ctas(const ts_ctx* c, int n_ctas, double prefill_block_pairs,
   for (int p = 0; p < n_ctas; p += 2) {
     const double d = (double)(n_ctas - p) * 148.0 / c->n_sms;
     int i = 1;
-    while (i < 7 && kSm[i] < d) ++i;
+    while (i < last && kSm[i] < d) ++i;
     const double rate = d >= 148.0 ? 1.0 : kRate[i - 1] + (kRate[i] - kRate[i - 1]) * (d - kSm[i - 1]) / (kSm[i] - kSm[i - 1]);
     const double td = t_dec_full / rate;
     const double t = std::max(td, (w_pf + (double)(n_ctas - p) * td) / n_ctas);

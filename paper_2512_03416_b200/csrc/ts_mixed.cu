@@ -24,8 +24,8 @@
 // next without a CTA-wide stop: the loaders run ahead into the next unit's K/V, its Q tiles land
 // as soon as the last Q K^T of the current unit has been issued, and its first Q K^T overlaps
 // the epilogue of the current unit.
-// The O rescale is lazy: a row's reference maximum only moves when the new maximum exceeds it by
-// more than 2^8, so most blocks never touch O.
+// The O rescale is lazy: a row's reference maximum only moves when a block's maximum exceeds it by
+// more than 2^8, so most blocks never touch O and take a single pass over their scores.
 // Every wait is bounded; a wait that runs out raises TS_DEV_TIMEOUT and the CTA drains.
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -227,11 +227,15 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// One row of a score block: p_i = 2^(v_i * scale + neg_m) for the 128 scores in v, written as bf16
-// pairs into TMEM columns [t_p, t_p + 64); returns the row sum of the unrounded p_i.
-__device__ __forceinline__ float exp_store(const float (&v)[128], float scale, float neg_m, uint32_t t_p) {
+// One row of a score block: p_i = 2^(x_i), x_i = v_i * scale + neg_m, for the 128 scores in v,
+// written as bf16 pairs into TMEM columns [t_p, t_p + 64); returns the row sum of the unrounded
+// p_i and, in x_max, the largest x_i. The maximum rides along in the issue slots the
+// special-function unit leaves free, so the common case needs no separate pass for it.
+__device__ __forceinline__ float exp_store(const float (&v)[128], float scale, float neg_m, uint32_t t_p,
+                                           float& x_max) {
   const uint64_t scale2 = pack_f2(scale, scale), negm2 = pack_f2(neg_m, neg_m);
   uint64_t sum_a = pack_f2(0.f, 0.f), sum_b = sum_a;
+  float xm0 = -CUDART_INF_F, xm1 = xm0, xm2 = xm0, xm3 = xm0;
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     uint32_t pk[16];
@@ -240,17 +244,21 @@ __device__ __forceinline__ float exp_store(const float (&v)[128], float scale, f
       const int e = c * 32 + 2 * i;
       float x0, x1;
       unpack_f2(fma2(pack_f2(v[e], v[e + 1]), scale2, negm2), x0, x1);
+      if ((i & 3) == 0) xm0 = max3(xm0, x0, x1);
+      else if ((i & 3) == 1) xm1 = max3(xm1, x0, x1);
+      else if ((i & 3) == 2) xm2 = max3(xm2, x0, x1);
+      else xm3 = max3(xm3, x0, x1);
       const float p0 = ex2(x0), p1 = ex2(x1);
       if (i & 1) sum_b = add2(sum_b, pack_f2(p0, p1)); else sum_a = add2(sum_a, pack_f2(p0, p1));
       pk[i] = pack2(p0, p1);
     }
     tmem_st16(t_p + c * 16, pk);
   }
+  x_max = fmaxf(fmaxf(xm0, xm1), fmaxf(xm2, xm3));
   float a0, a1;
   unpack_f2(add2(sum_a, sum_b), a0, a1);
   return a0 + a1;
 }
-
 
 // One prefill work unit as its claimer publishes it in shared memory (8 words), and the shape
 // every role derives from it.
@@ -412,42 +420,52 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
           for (int i = 0; i < 128; ++i)
             if (i >= nvalid) v[i] = -CUDART_INF_F;             // 2^(-inf) = 0 exactly
         }
-        // row maximum of the raw scores (the scale is positive, so it commutes with max)
-        float m0 = max3(v[0], v[1], v[2]), m1 = max3(v[3], v[4], v[5]);
-        float m2 = max3(v[6], v[7], v[8]), m3 = max3(v[9], v[10], v[11]);
+        // p = 2^(s*scale - m_ref) as bf16 over the first 64 columns of S (the scores are in
+        // registers), against the reference the row already has: the result is exact for any
+        // common reference, and p <= 2^threshold keeps the bf16 P and the fp32 sums comfortable.
+        // Only a row whose block maximum exceeds its reference by more than the threshold (always
+        // on a unit's first block, seldom afterwards) moves the reference, rescales O and redoes
+        // the block.
+        float x_max = CUDART_INF_F, ls = 0.f;
+        if (j > 0) ls = exp_store(v, scale, -m_ref, tS, x_max);
+        const bool move = x_max > kRescaleThreshold;
+        if (__any_sync(0xffffffffu, move)) {
+          float alpha = 1.f;
+          if (j == 0) {
+            // row maximum of the raw scores (the scale is positive, so it commutes with max)
+            float m0 = max3(v[0], v[1], v[2]), m1 = max3(v[3], v[4], v[5]);
+            float m2 = max3(v[6], v[7], v[8]), m3 = max3(v[9], v[10], v[11]);
 #pragma unroll
-        for (int i = 12; i < 124; i += 8) {
-          m0 = max3(m0, v[i], v[i + 1]);
-          m1 = max3(m1, v[i + 2], v[i + 3]);
-          m2 = max3(m2, v[i + 4], v[i + 5]);
-          m3 = max3(m3, v[i + 6], v[i + 7]);
-        }
-        m0 = max3(m0, v[124], v[125]);
-        m1 = max3(m1, v[126], v[127]);
-        const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * scale;
-        // lazy rescale: move the reference maximum only when it is exceeded by 2^threshold
-        const bool move = mx > m_ref + kRescaleThreshold;   // first block: m_ref = -inf, so true
-        float alpha = 1.f;
-        if (move) {
-          alpha = ex2(m_ref - mx);                          // 0 on the first block
-          m_ref = mx;
-          l *= alpha;
-        }
-        if (j > 0 && __any_sync(0xffffffffu, move)) {
-          wait(BAR_O_FULL + x, (sx + j - 1) & 1);           // P V of block j-1 has landed in O
-          tc_fence_after();
+            for (int i = 12; i < 124; i += 8) {
+              m0 = max3(m0, v[i], v[i + 1]);
+              m1 = max3(m1, v[i + 2], v[i + 3]);
+              m2 = max3(m2, v[i + 4], v[i + 5]);
+              m3 = max3(m3, v[i + 6], v[i + 7]);
+            }
+            m0 = max3(m0, v[124], v[125]);
+            m1 = max3(m1, v[126], v[127]);
+            m_ref = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * scale;
+          } else {
+            if (move) {
+              alpha = ex2(-x_max);                            // 2^(old reference - new reference)
+              m_ref += x_max;
+              l *= alpha;
+            }
+            wait(BAR_O_FULL + x, (sx + j - 1) & 1);           // P V of block j-1 has landed in O
+            tc_fence_after();
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            float ov[32];
-            tmem_ld32(ov, tO + c * 32);
-            tmem_ld_wait();
+            for (int c = 0; c < 4; ++c) {
+              float ov[32];
+              tmem_ld32(ov, tO + c * 32);
+              tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) ov[i] *= alpha;
-            tmem_st32(tO + c * 32, ov);
+              for (int i = 0; i < 32; ++i) ov[i] *= alpha;
+              tmem_st32(tO + c * 32, ov);
+            }
           }
+          ls = exp_store(v, scale, -m_ref, tS, x_max);
         }
-        // p = 2^(s*scale - m_ref) as bf16 over the first 64 columns of S (the scores are in registers)
-        l += exp_store(v, scale, -m_ref, tS);
+        l += ls;
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(bar(BAR_P_FULL + x));
