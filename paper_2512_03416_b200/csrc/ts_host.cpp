@@ -496,8 +496,12 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
     c->prof_mixed.push_back(0);
     TS_CUDA(c, cudaEventRecord(pe[0], stream));
   }
-  TS_CUDA(c, ts::launch_kv_append(d, stream));
-  ++c->cnt.kernel_launches;
+  // head_dim 128 steps with prefill tiles: the mixed kernel appends the new K/V itself
+  const bool append_in_kernel = attention && c->n_prefill_items > 0 && c->cfg.head_dim == 128;
+  if (!append_in_kernel) {
+    TS_CUDA(c, ts::launch_kv_append(d, stream));
+    ++c->cnt.kernel_launches;
+  }
   if (attention) {
     if (pe) TS_CUDA(c, cudaEventRecord(pe[1], stream));
     d.n_prefill_items = c->n_prefill_items;
@@ -860,7 +864,10 @@ int ts_last_device_status(ts_ctx* c, void* cuda_stream, int32_t* status_out) {
   if (!c->status_cleared) return TS_OK;  // nothing has run yet
   int32_t* dev = (int32_t*)((char*)c->cfg.workspace + c->L.off_status);
   TS_CUDA(c, cudaMemcpyAsync(status_out, dev, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
-  TS_CUDA(c, cudaMemsetAsync(dev, 0, sizeof(int32_t), stream));
+  TS_CUDA(c, cudaStreamSynchronize(stream));
+  // a clean status clears only its word; after a failure the kernels' counters next to it may be
+  // stale as well, so the whole block goes back to zero
+  TS_CUDA(c, cudaMemsetAsync(dev, 0, *status_out ? kAlign : sizeof(int32_t), stream));
   TS_CUDA(c, cudaStreamSynchronize(stream));
   return (*status_out & TS_DEV_TIMEOUT) ? TS_ERR_DEVICE_TIMEOUT : TS_OK;
 }

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "../../include/tokenscale.h"
+
 #include <utility>
 
 namespace ts {
@@ -48,8 +50,10 @@ struct StepDevice {
   uint16_t* pool;          // caller's KV pool
   int32_t* table;          // [max_requests][max_pages_per_req]
   int32_t* status;         // device status word
-  int32_t* pf_queue;       // [0] next prefill work unit of the step, [1] decode CTAs of the mixed
-                           // kernel that have finished their units (both zeroed by the append kernel)
+  int32_t* pf_queue;       // counters of the mixed kernel, all zero between launches (its last CTA
+                           // to leave resets them): [0] next prefill work unit, [1] decode CTAs
+                           // that have finished their units, [2] CTAs that have appended their
+                           // share of the new tokens, [3] CTAs that have left
   float* part_acc;         // [max_partials][Hq][D]
   float* part_ml;          // [max_partials][Hq][2]  (running max in log2 units, sum)
   // per step (device meta area)
@@ -81,7 +85,8 @@ cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream);
 // through kv_map (5-D view of the pool: head_dim, slot, KV head, K|V, page; box 64 x 16 x 1 x 2 x 1).
 // Prefill tiles items[0, n_prefill_items), head_dim 128: persistent tcgen05/TMEM kernel of n_ctas
 // CTAs. The first n_prefill_ctas CTAs work on the prefill queue only; the others first run all
-// decode splits (as launch_decode would, needs G <= 8) and then join the prefill queue. With
+// decode splits (as launch_decode would, needs G <= 8) and then join the prefill queue. The
+// kernel also appends the step's new K/V itself (no launch_kv_append before it). With
 // n_prefill_ctas == n_ctas the decode splits are left to launch_decode. When it runs the decode
 // splits it also merges them (no launch_combine needed).
 // q_map views q as (head_dim, G, KV head, token), box 64 x G x 1 x 128/G.
@@ -110,6 +115,76 @@ inline cudaError_t launch_pdl(void (*kernel)(Params...), dim3 grid, dim3 block, 
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 #ifdef __CUDACC__
+// Copies the K/V of the step's new tokens into their pages (Sec. 2.1): one warp per token at a time,
+// warps `first_warp`, `first_warp + n_warps`, ... of the launch; a lane moves 16-byte chunks, eight
+// loads in flight before the first store, and the source loads are issued before the block-table
+// look-up they do not depend on. `rows` = a shared-memory copy of the step's row arrays made by
+// stage_rows (the token -> row search and the row's slot and length then cost no global round trips).
+// Slots and page ids are range checked; a bad one sets a status bit and skips the token.
+__device__ __forceinline__ void stage_rows(const StepDevice& s, int32_t* rows, int tid, int n_threads) {
+  const int n = s.n_rows + 1;                  // rows[0..n): first-token prefix sums, then ctx, then slot
+  for (int i = tid; i < n; i += n_threads) {
+    rows[i] = s.row_tok0[i];
+    if (i < s.n_rows) {
+      rows[n + i] = s.row_ctx[i];
+      rows[2 * n + i] = s.row_slot[i];
+    }
+  }
+}
+__host__ __device__ inline size_t staged_rows_bytes(int n_rows) { return (size_t)3 * (n_rows + 1) * sizeof(int32_t); }
+__device__ __forceinline__ void append_tokens(const StepDevice& s, const int32_t* rows, int first_warp, int n_warps,
+                                              int lane) {
+  const int n = s.n_rows + 1;
+  const int32_t* row_start = rows;
+  const int cpr = s.D / 8;                      // chunks per (token, head) row
+  const int per_tok = 2 * s.Hkv * cpr;
+  for (int tok = first_warp; tok < s.n_tokens; tok += n_warps) {
+    int lo = 0, hi = s.n_rows;                  // row of this token: last r with row_start[r] <= tok
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (row_start[mid] <= tok) lo = mid; else hi = mid;
+    }
+    const int t = rows[n + lo] + (tok - row_start[lo]);
+    const int slot = rows[2 * n + lo];
+    const bool index_ok = (unsigned)slot < (unsigned)s.max_requests && (unsigned)(t >> 4) < (unsigned)s.max_pages_per_req;
+    int page = -1;
+    for (int base = 0; base < per_tok; base += 256) {
+      uint4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c = base + u * 32 + lane;
+        if (c < per_tok) {
+          const int kv = c / (s.Hkv * cpr);
+          const int rem = c - kv * s.Hkv * cpr;
+          const int head = rem / cpr, ch = rem % cpr;
+          v[u] = *reinterpret_cast<const uint4*>((kv ? s.v_new : s.k_new) + ((size_t)tok * s.Hkv + head) * s.D + ch * 8);
+        }
+      }
+      if (base == 0) {
+        if (!index_ok) {
+          if (lane == 0) atomicOr(s.status, TS_DEV_BAD_INDEX);
+          break;
+        }
+        page = s.table[(size_t)slot * s.max_pages_per_req + (t >> 4)];
+        if ((unsigned)page >= (unsigned)s.n_pages) {
+          if (lane == 0) atomicOr(s.status, TS_DEV_BAD_PAGE);
+          break;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c = base + u * 32 + lane;
+        if (c < per_tok) {
+          const int kv = c / (s.Hkv * cpr);
+          const int rem = c - kv * s.Hkv * cpr;
+          const int head = rem / cpr, ch = rem % cpr;
+          uint16_t* dst = s.pool + ((((size_t)page * 2 + kv) * s.Hkv + head) * kPageSize + (t & 15)) * s.D + ch * 8;
+          *reinterpret_cast<uint4*>(dst) = v[u];
+        }
+      }
+    }
+  }
+}
 // Log-sum-exp merge of the splits of one (token, head) for head_dim element d: the exact merge
 //   m = max m_i,  l = sum l_i 2^(m_i - m),  O = sum acc_i 2^(m_i - m) / l
 // over the partial slots [first_partial, first_partial + n_splits). Eight splits' loads are in

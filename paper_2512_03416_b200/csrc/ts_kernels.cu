@@ -71,65 +71,16 @@ __global__ void table_update_kernel(int32_t* table, int width, int max_requests,
   table[(size_t)d.slot * width + d.index] = d.page;
 }
 
-// One warp per new token at a time (grid-stride over tokens): its lanes copy the token's
-// 2 * Hkv * D / 8 sixteen-byte chunks of K and V, eight loads in flight per lane before the first
-// store. The row prefix sums sit in shared memory, so the token -> row search costs no global
-// round trips, and a block's warps overlap one another's table look-ups.
+// KV append as a launch of its own (ts_kv_append, and steps whose attention kernel does not
+// append itself): one warp per new token at a time, see append_tokens.
 __global__ void kv_append_kernel(StepDevice s) {
-  extern __shared__ int32_t row_start[];        // [n_rows + 1]
+  extern __shared__ int32_t rows[];             // staged row arrays, see stage_rows
   pdl_launch_dependents();
   pdl_wait();
-  if (blockIdx.x == 0 && threadIdx.x == 0 && s.pf_queue) {   // the step's work queue and decode-done count
-    s.pf_queue[0] = 0;
-    s.pf_queue[1] = 0;
-  }
-  for (int i = threadIdx.x; i <= s.n_rows; i += blockDim.x) row_start[i] = s.row_tok0[i];
+  stage_rows(s, rows, threadIdx.x, blockDim.x);
   __syncthreads();
   const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int cpr = s.D / 8;                      // chunks per (token, head) row
-  const int per_tok = 2 * s.Hkv * cpr;
-  for (int tok = blockIdx.x * warps + warp; tok < s.n_tokens; tok += gridDim.x * warps) {
-    int lo = 0, hi = s.n_rows;                  // row of this token: last r with row_start[r] <= tok
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (row_start[mid] <= tok) lo = mid; else hi = mid;
-    }
-    const int t = s.row_ctx[lo] + (tok - row_start[lo]);
-    const int slot = s.row_slot[lo];
-    if ((unsigned)slot >= (unsigned)s.max_requests || (unsigned)(t >> 4) >= (unsigned)s.max_pages_per_req) {
-      if (lane == 0) atomicOr(s.status, TS_DEV_BAD_INDEX);
-      continue;
-    }
-    const int page = s.table[(size_t)slot * s.max_pages_per_req + (t >> 4)];
-    if ((unsigned)page >= (unsigned)s.n_pages) {
-      if (lane == 0) atomicOr(s.status, TS_DEV_BAD_PAGE);
-      continue;
-    }
-    for (int base = 0; base < per_tok; base += 256) {
-      uint4 v[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int c = base + u * 32 + lane;
-        if (c < per_tok) {
-          const int kv = c / (s.Hkv * cpr);
-          const int rem = c - kv * s.Hkv * cpr;
-          const int head = rem / cpr, ch = rem % cpr;
-          v[u] = *reinterpret_cast<const uint4*>((kv ? s.v_new : s.k_new) + ((size_t)tok * s.Hkv + head) * s.D + ch * 8);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int c = base + u * 32 + lane;
-        if (c < per_tok) {
-          const int kv = c / (s.Hkv * cpr);
-          const int rem = c - kv * s.Hkv * cpr;
-          const int head = rem / cpr, ch = rem % cpr;
-          uint16_t* dst = s.pool + ((((size_t)page * 2 + kv) * s.Hkv + head) * kPageSize + (t & 15)) * s.D + ch * 8;
-          *reinterpret_cast<uint4*>(dst) = v[u];
-        }
-      }
-    }
-  }
+  append_tokens(s, rows, blockIdx.x * warps + warp, gridDim.x * warps, lane);
 }
 
 // Merge of the splits of one token: grid (n_combines, Hq), block D threads.
@@ -438,7 +389,7 @@ cudaError_t launch_kv_append(const StepDevice& s, cudaStream_t stream) {
   const int threads = 256;                                    // eight warps = eight tokens per block at a time
   const int blocks = (s.n_tokens + 7) / 8;
   const int grid = blocks < 148 * 8 ? blocks : 148 * 8;
-  return launch_pdl(kv_append_kernel, dim3(grid), dim3(threads), (s.n_rows + 1) * sizeof(int32_t), stream, s);
+  return launch_pdl(kv_append_kernel, dim3(grid), dim3(threads), staged_rows_bytes(s.n_rows), stream, s);
 }
 
 cudaError_t launch_attention(const StepDevice& s, cudaStream_t stream) {

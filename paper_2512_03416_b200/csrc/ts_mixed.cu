@@ -26,6 +26,8 @@
 // the epilogue of the current unit.
 // The O rescale is lazy: a row's reference maximum only moves when a block's maximum exceeds it by
 // more than 2^8, so most blocks never touch O and take a single pass over their scores.
+// The kernel starts by appending the step's new K/V to the pages itself (every CTA a share of
+// the tokens, then a launch-wide counter barrier), which saves a launch in front of it.
 // Every wait is bounded; a wait that runs out raises TS_DEV_TIMEOUT and the CTA drains.
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -362,21 +364,44 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
     tc_fence_before();
     cta_sync();
     tc_fence_after();
-    if (!decode_first) pdl_wait();   // set-up done; from here on the pool, tables and Q are read
   };
   // Decode-first CTAs: warps 0-7 run the CTA's decode units, the other warps wait for them.
   auto decode_phase_idle = [&]() {
-    if (decode_first) {
-      pdl_wait();
-      cta_sync();
-    }
+    if (decode_first) cta_sync();
   };
+
+  // ---------------------------------------------------------------- KV append (Sec. 2.1)
+  // Every CTA copies its share of the step's new tokens into their pages, then all CTAs of the
+  // launch meet at a counter (they are all resident: one per SM), so that the attention below
+  // sees every page complete. This replaces a launch of its own in front of the kernel.
+  pdl_wait();                  // the previous step's kernels are done with the pool and the counters
+  {
+    int32_t* rows = reinterpret_cast<int32_t*>(smem);   // the window's start is free until the roles begin
+    stage_rows(s, rows, tid, kPfThreads);
+    cta_sync();
+    append_tokens(s, rows, (int)blockIdx.x * (kPfThreads / 32) + warp, (int)gridDim.x * (kPfThreads / 32), lane);
+    __threadfence();           // this thread's page writes are visible before the CTA counts itself
+    fence_proxy_async();       // and the scratch is handed on to the roles' copies
+    cta_sync();
+    if (tid == 0) {
+      atomicAdd(s.pf_queue + 2, 1);
+      const volatile int32_t* arrived = s.pf_queue + 2;
+      const long long t0 = clock64();
+      while (*arrived < (int)gridDim.x) {
+        if (clock64() - t0 > kWaitCycles) {
+          atomicOr(s.status, TS_DEV_TIMEOUT);
+          break;
+        }
+      }
+      __threadfence();
+    }
+    cta_sync();
+  }
 
   if (warp < 8) {
     // ------------------------------------------ softmax + epilogue: thread = query row of tile x
     reg_inc<kRegsSoftmax>();
     if (decode_first) {
-      pdl_wait();
       dec::decode_units<128, 1, 3>(s, &kv_map, smem, base, (int)blockIdx.x - n_prefill_ctas,
                                    (int)gridDim.x - n_prefill_ctas);
       if (tid == 0) {          // this CTA's split partials are written: count it as done
@@ -779,6 +804,16 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
   tc_fence_before();
   cta_sync();
   if (warp == kWarpMma) tmem_dealloc(misc[0], 512);
+  if (tid == 0) {
+    // the last CTA to leave puts the launch's counters back to zero for the next launch
+    __threadfence();
+    if (atomicAdd(s.pf_queue + 3, 1) == (int)gridDim.x - 1) {
+      s.pf_queue[0] = 0;
+      s.pf_queue[1] = 0;
+      s.pf_queue[2] = 0;
+      s.pf_queue[3] = 0;
+    }
+  }
 }
 
 }  // namespace
