@@ -34,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the workload's dominant kernel, from
 # the ncu captures summarised under profiles/ (decode_kernel on config2, mixed_kernel on config3).
 # An entry is dropped (null in the output) when its kernel has changed since the capture.
-KERNEL_TRAFFIC_BYTES = {"config2": 7.795e8, "config3": 8.257e8}
+KERNEL_TRAFFIC_BYTES = {"config2": 7.755e8, "config3": 8.413e8}
 
 WORKLOADS = {
     "config2": (wl.config2, "decode-only batch, 8B-shaped layer (64 decode rows, ctx lognormal median 2048)"),
@@ -256,7 +256,7 @@ def rooflines(peaks, peak_kind, flops, byts, step_ms, prof, parts, traffic=None)
     `parts` holds algorithmic work per recorded step, averaged over all recorded steps:
     dec_bytes of the steps whose decode rows ran in decode_kernel, pf_flops of the steps whose launch
     held prefill tiles only, and mixed_bytes / mixed_flops of the steps where one launch ran tiles
-    and decode rows together (that launch does everything but the append kernel's page writes).
+    and decode rows together (that launch is the whole step: append, attention, split merge).
     The dominant kernel is the one with the largest total time; achieved = its algorithmic work
     over its own time.
     """
@@ -337,7 +337,7 @@ def run_static(args, world, rank, local, barrier):
                                             zip(batch.ctx_len[~dec].tolist(), batch.q_len[~dec].tolist())))
     mixed = prof.get("mixed_steps", 0) > 0          # one launch ran the tiles and the decode rows together
     parts = {"dec_bytes": 0.0 if mixed else dec_bytes, "pf_flops": 0.0 if mixed else pf_flops,
-             "mixed_bytes": byts - batch.n_tokens * s.kv_bytes_per_token if mixed else 0.0,
+             "mixed_bytes": byts if mixed else 0.0,     # the mixed launch also appends the new K/V
              "mixed_flops": flops if mixed else 0.0}
 
     # end to end: host buffers in, host buffer out, through ts_mixed_step_host
@@ -417,9 +417,8 @@ def run_replay(args, world, rank, local, barrier):
     dec_bytes = pf_flops = mixed_bytes = mixed_flops = 0.0
     for ps, w in zip(run.steps, work):
         n_dec = sum(1 for t in ps.q_len if t == 1)
-        n_new = int(sum(ps.q_len))
         if ps.prefill_tokens > 0 and n_dec > 0:
-            mixed_bytes += w[1] - n_new * s.kv_bytes_per_token
+            mixed_bytes += w[1]                      # the mixed launch also appends the new K/V
             mixed_flops += w[0]
         elif ps.prefill_tokens > 0:
             pf_flops += w[0]
