@@ -203,6 +203,11 @@ int ts_kv_append(ts_ctx* ctx, const ts_step* step, void* cuda_stream);
  * writes out. Everything is enqueued on cuda_stream; the call does not synchronise.
  * Enforces Sec. 4.4's budget: (prefill tokens + decode rows) <= chunk_size, else TS_ERR_BUDGET.
  * Updates the Token Velocity counters. An empty step (n_rows == 0) is TS_OK and launches nothing.
+ * A step with prefill rows runs as one kernel that fills every SM and whose thread blocks wait
+ * for one another (bounded waits): steps of different contexts on the same device must not
+ * overlap on the GPU -- issue them to one stream, or order the streams with events. If they do
+ * overlap, the waits run out, the step's output is wrong and ts_last_device_status reports
+ * TS_DEV_TIMEOUT; nothing hangs.
  */
 int ts_mixed_step(ts_ctx* ctx, const ts_step* step, void* cuda_stream);
 
