@@ -11,6 +11,8 @@ Plain restatements of the paper's counting rules, used to check the library's co
 * Sec. 4.4: chunk size bounds (prefill tokens + decode batch size) of one iteration;
   Eq. 5: V_D^{P'} = (chunk_size - batch_size) / TPOT_SLO.
 * Eq. 6: Mem_Reserved = V_D^{P'} * Mem_T * TTFT_SLO.
+* Sec. 4.4, chunk-size selection: the iteration time is profiled while the prefill chunk grows,
+  until the TPOT SLO is violated; the chunk size chosen is the largest one before that.
 """
 from __future__ import annotations
 
@@ -41,6 +43,28 @@ def convertible_prefill_velocity(chunk_size: int, batch_size: float, tpot_slo_s:
 def reserved_memory(v_dp: float, mem_per_token: float, ttft_slo_s: float) -> float:
     """Eq. 6."""
     return v_dp * mem_per_token * ttft_slo_s
+
+
+def reserved_tokens(v_dp: float, ttft_slo_s: float) -> float:
+    """Eq. 6 divided by the per-token footprint Mem_T: the tokens' worth of memory held back."""
+    return v_dp * ttft_slo_s
+
+
+def reserved_pages(v_dp: float, ttft_slo_s: float, page_size: int) -> int:
+    """Eq. 6 in whole KV pages."""
+    return int(math.ceil(reserved_tokens(v_dp, ttft_slo_s) / page_size))
+
+
+def pick_chunk_size(prefill_tokens, iteration_seconds, decode_batch_size: int, tpot_slo_s: float) -> int:
+    """Sec. 4.4: walk the profile in the order it was taken (growing prefill chunk) and stop at
+    the first iteration time above the TPOT SLO; chunk size = the last prefill size before that
+    plus the decode batch size (the definition of chunk size), 0 if even the first point is late."""
+    best = 0
+    for t, sec in zip(prefill_tokens, iteration_seconds):
+        if sec > tpot_slo_s:
+            break
+        best = int(t) + int(decode_batch_size)
+    return best
 
 
 @dataclass

@@ -307,6 +307,26 @@ def pin_fig7_worked_example():
         assert velocity.request_policy_fires(int(n_req), float(thr)) == bool(int(exp_fire))
 
 
+def pin_chunk_size_selection():
+    """Sec. 4.4 against a closed form: with an iteration time that is affine in the prefill
+    tokens, a + b*T, the largest admissible T is floor((SLO - a) / b) on a unit grid."""
+    a, b, slo, batch = 0.004, 1.0e-5, 0.1, 64
+    grid = list(range(0, 20001, 250))
+    secs = [a + b * t for t in grid]
+    t_max = int(math.floor((slo - a) / b / 250.0 + 1e-9)) * 250
+    assert velocity.pick_chunk_size(grid, secs, batch, slo) == t_max + batch == 9500 + 64
+    # stops at the FIRST violation: a later point that happens to be fast again does not count
+    assert velocity.pick_chunk_size([128, 256, 512, 1024], [0.02, 0.2, 0.03, 0.04], 10, 0.1) == 138
+    assert velocity.pick_chunk_size([128, 256], [0.2, 0.01], 10, 0.1) == 0
+    assert velocity.pick_chunk_size([], [], 10, 0.1) == 0
+    # Eq. 6 in pages: velocity * TTFT_SLO tokens, rounded up to 16-token pages
+    v = velocity.convertible_prefill_velocity(9564, 64, 0.1)             # 95,000 tokens/s
+    assert abs(v - 95000.0) < 1e-6
+    assert abs(velocity.reserved_tokens(v, 0.25) - 23750.0) < 1e-6
+    assert velocity.reserved_pages(v, 0.25, 16) == 1485                   # ceil(23750 / 16)
+    assert abs(velocity.reserved_memory(v, 4096.0, 0.25) - velocity.reserved_tokens(v, 0.25) * 4096.0) < 1e-3
+
+
 def pin_eq5_eq6_and_counters():
     assert velocity.prefill_budget(8448, 256) == 8192
     assert velocity.prefill_budget(100, 256) == 0
@@ -328,7 +348,7 @@ PINS = [pin_single_key_returns_its_value, pin_two_keys_logistic_weights,
         pin_table_permutation_invariance, pin_decode_equals_last_prefill_row,
         pin_chunked_equals_unchunked, pin_softmax_weights_and_convexity, pin_gqa_group_symmetry,
         pin_needle_visibility, pin_every_position_is_gathered_from_its_slot,
-        pin_append_writes_exactly_the_live_slots, pin_fig7_worked_example, pin_eq5_eq6_and_counters]
+        pin_append_writes_exactly_the_live_slots, pin_fig7_worked_example, pin_eq5_eq6_and_counters, pin_chunk_size_selection]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=[p.__name__ for p in PINS])
