@@ -266,6 +266,33 @@ int ts_profile_read(ts_ctx* ctx, void* cuda_stream, ts_profile* out);
 int32_t ts_prefill_budget(const ts_ctx* ctx, int32_t decode_batch_size);
 
 /*
+ * Configuring a Convertible Decoder (Sec. 4.4). Host-only arithmetic, no context needed.
+ *
+ * ts_pick_chunk_size: the chunk size is found by profiling the iteration time while the prefill
+ * chunk grows, until the TPOT SLO is violated; the largest chunk size before that is taken.
+ * prefill_tokens[i] (ascending, > 0) are the profiled prefill sizes at a fixed decode batch,
+ * iteration_seconds[i] the caller's iteration time at each (e.g. the measured ts_mixed_step
+ * time times the number of layers). Returns prefill_tokens[last point within the SLO before the
+ * first violation] + decode_batch_size -- chunk size is defined as prefill tokens + decode batch
+ * size -- or 0 when the first point already violates it, or TS_ERR_INVALID (negative) for null
+ * arrays, n <= 0, sizes that are not ascending, a negative batch size or a non-positive SLO.
+ *
+ * ts_convertible_prefill_velocity: Eq. 5, V_D^{P'} = (chunk_size - batch_size) / TPOT_SLO in
+ * tokens/s, with the average decode batch size as a real number; 0 when the batch fills the chunk
+ * or the SLO is not positive.
+ *
+ * ts_reserved_memory: Eq. 6, Mem_Reserved = V_D^{P'} * Mem_T * TTFT_SLO in the unit of
+ * mem_per_token. ts_reserved_pages: the same in whole KV pages of page_size tokens (Mem_T cancels:
+ * V_D^{P'} * TTFT_SLO tokens, rounded up) -- the value for ts_config.reserved_pages. Both return
+ * 0 for non-positive arguments.
+ */
+int32_t ts_pick_chunk_size(const int32_t* prefill_tokens, const double* iteration_seconds, int32_t n,
+                           int32_t decode_batch_size, double tpot_slo_s);
+double ts_convertible_prefill_velocity(int32_t chunk_size, double decode_batch_size, double tpot_slo_s);
+double ts_reserved_memory(double prefill_velocity, double mem_per_token, double ttft_slo_s);
+int32_t ts_reserved_pages(double prefill_velocity, double ttft_slo_s, int32_t page_size);
+
+/*
  * ts_plan_step: host-only. Validates the step exactly as ts_mixed_step does and writes the
  * work list it would launch: one record of 8 int32 per work item
  *   {row, kind (0 decode split, 1 prefill tile), q_begin, q_count, k_begin, k_end,

@@ -67,7 +67,8 @@ EXPORTS = ["ts_pool_bytes", "ts_workspace_bytes", "ts_create", "ts_destroy", "ts
            "ts_request_set_len", "ts_kv_append", "ts_mixed_step", "ts_mixed_step_host",
            "ts_velocity", "ts_report_step_time", "ts_prefill_budget", "ts_plan_step",
            "ts_last_device_status", "ts_last_cuda_error", "ts_strerror", "ts_profile_enable",
-           "ts_profile_read", "ts_decode_attention_static", "ts_alloc_step"]
+           "ts_profile_read", "ts_decode_attention_static", "ts_alloc_step", "ts_pick_chunk_size",
+           "ts_convertible_prefill_velocity", "ts_reserved_memory", "ts_reserved_pages"]
 
 _lib = None
 
@@ -108,6 +109,15 @@ def lib() -> ctypes.CDLL:
         L.ts_prefill_budget.restype = ctypes.c_int32
         L.ts_prefill_budget.argtypes = [vp, ctypes.c_int32]
         L.ts_plan_step.argtypes = [vp, stepp, _i32p, ctypes.c_int32, _i32p]
+        L.ts_pick_chunk_size.restype = ctypes.c_int32
+        L.ts_pick_chunk_size.argtypes = [_i32p, ctypes.POINTER(ctypes.c_double), ctypes.c_int32, ctypes.c_int32,
+                                         ctypes.c_double]
+        L.ts_convertible_prefill_velocity.restype = ctypes.c_double
+        L.ts_convertible_prefill_velocity.argtypes = [ctypes.c_int32, ctypes.c_double, ctypes.c_double]
+        L.ts_reserved_memory.restype = ctypes.c_double
+        L.ts_reserved_memory.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double]
+        L.ts_reserved_pages.restype = ctypes.c_int32
+        L.ts_reserved_pages.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_int32]
         L.ts_last_device_status.argtypes = [vp, vp, _i32p]
         L.ts_last_cuda_error.argtypes = [vp]
         L.ts_profile_enable.argtypes = [vp, ctypes.c_int]
@@ -226,6 +236,25 @@ def ts_report_step_time(ctx, seconds: float) -> int:
 
 def ts_prefill_budget(ctx, decode_batch_size: int) -> int:
     return lib().ts_prefill_budget(ctx, decode_batch_size)
+
+
+def ts_pick_chunk_size(prefill_tokens, iteration_seconds, decode_batch_size: int, tpot_slo_s: float) -> int:
+    n = len(prefill_tokens)
+    a = (ctypes.c_int32 * max(n, 1))(*[int(t) for t in prefill_tokens])
+    b = (ctypes.c_double * max(n, 1))(*[float(t) for t in iteration_seconds])
+    return lib().ts_pick_chunk_size(a, b, n, decode_batch_size, tpot_slo_s)
+
+
+def ts_convertible_prefill_velocity(chunk_size: int, decode_batch_size: float, tpot_slo_s: float) -> float:
+    return lib().ts_convertible_prefill_velocity(chunk_size, decode_batch_size, tpot_slo_s)
+
+
+def ts_reserved_memory(prefill_velocity: float, mem_per_token: float, ttft_slo_s: float) -> float:
+    return lib().ts_reserved_memory(prefill_velocity, mem_per_token, ttft_slo_s)
+
+
+def ts_reserved_pages(prefill_velocity: float, ttft_slo_s: float, page_size: int = 16) -> int:
+    return lib().ts_reserved_pages(prefill_velocity, ttft_slo_s, page_size)
 
 
 def ts_plan_step(ctx, step: ts_step):

@@ -835,6 +835,38 @@ int32_t ts_prefill_budget(const ts_ctx* c, int32_t decode_batch_size) {
   return std::max(c->cfg.chunk_size - decode_batch_size, 0);
 }
 
+int32_t ts_pick_chunk_size(const int32_t* prefill_tokens, const double* iteration_seconds, int32_t n,
+                           int32_t decode_batch_size, double tpot_slo_s) {
+  if (!prefill_tokens || !iteration_seconds || n <= 0 || decode_batch_size < 0 || !(tpot_slo_s > 0.0))
+    return TS_ERR_INVALID;
+  for (int i = 0; i < n; ++i) {
+    if (prefill_tokens[i] <= 0 || (i > 0 && prefill_tokens[i] <= prefill_tokens[i - 1])) return TS_ERR_INVALID;
+    if (!(iteration_seconds[i] >= 0.0)) return TS_ERR_INVALID;
+  }
+  int32_t best = 0;
+  for (int i = 0; i < n; ++i) {                 // the profile stops counting at the first violation
+    if (iteration_seconds[i] > tpot_slo_s) break;
+    best = prefill_tokens[i] + decode_batch_size;
+  }
+  return best;
+}
+
+double ts_convertible_prefill_velocity(int32_t chunk_size, double decode_batch_size, double tpot_slo_s) {
+  if (!(tpot_slo_s > 0.0) || !(decode_batch_size >= 0.0) || (double)chunk_size <= decode_batch_size) return 0.0;
+  return ((double)chunk_size - decode_batch_size) / tpot_slo_s;
+}
+
+double ts_reserved_memory(double prefill_velocity, double mem_per_token, double ttft_slo_s) {
+  if (!(prefill_velocity > 0.0) || !(mem_per_token > 0.0) || !(ttft_slo_s > 0.0)) return 0.0;
+  return prefill_velocity * mem_per_token * ttft_slo_s;
+}
+
+int32_t ts_reserved_pages(double prefill_velocity, double ttft_slo_s, int32_t page_size) {
+  if (!(prefill_velocity > 0.0) || !(ttft_slo_s > 0.0) || page_size <= 0) return 0;
+  const double pages = std::ceil(prefill_velocity * ttft_slo_s / (double)page_size - 1e-9);
+  return pages > 2147483647.0 ? 2147483647 : (int32_t)pages;
+}
+
 int ts_plan_step(ts_ctx* c, const ts_step* st, int32_t* items, int32_t items_capacity,
                  int32_t* n_items_out) {
   if (!n_items_out) return TS_ERR_INVALID;

@@ -257,3 +257,29 @@ def test_counters_match_the_oracle_mirror():
     assert B.ts_prefill_budget(h, 28) == velocity.prefill_budget(128, 28) == 100       # Eq. 5 numerator
     assert B.ts_prefill_budget(h, 500) == 0
     B.ts_destroy(h)
+
+
+def test_convertible_decoder_configuration_matches_the_oracle():
+    """Sec. 4.4 / Eq. 5 / Eq. 6 through the C ABI against oracle/velocity.py on seeded profiles."""
+    rng = np.random.Generator(np.random.Philox(44))
+    for _ in range(200):
+        n = int(rng.integers(1, 12))
+        sizes = np.cumsum(rng.integers(1, 2000, size=n)).astype(np.int32)
+        secs = np.sort(rng.uniform(0.0, 0.2, size=n))
+        if rng.random() < 0.3:                       # a noisy profile: not monotone
+            secs = rng.permutation(secs)
+        batch, slo = int(rng.integers(0, 300)), float(rng.uniform(0.01, 0.2))
+        got = B.ts_pick_chunk_size(sizes.tolist(), secs.tolist(), batch, slo)
+        assert got == velocity.pick_chunk_size(sizes.tolist(), secs.tolist(), batch, slo)
+        v = B.ts_convertible_prefill_velocity(max(got, 1), float(batch) / 2, slo)
+        assert abs(v - max(velocity.convertible_prefill_velocity(max(got, 1), batch / 2, slo), 0.0)) <= 1e-9 * max(v, 1.0)
+        ttft = float(rng.uniform(0.05, 2.0))
+        assert abs(B.ts_reserved_memory(v, 4096.0, ttft) - (velocity.reserved_memory(v, 4096.0, ttft) if v > 0 else 0.0)) <= 1e-6 * max(v, 1.0)
+        assert B.ts_reserved_pages(v, ttft, 16) == (velocity.reserved_pages(v, ttft, 16) if v > 0 else 0)
+    # invalid profiles
+    assert B.ts_pick_chunk_size([], [], 4, 0.1) == B.TS_ERR_INVALID
+    assert B.ts_pick_chunk_size([256, 128], [0.01, 0.02], 4, 0.1) == B.TS_ERR_INVALID      # not ascending
+    assert B.ts_pick_chunk_size([128], [0.01], -1, 0.1) == B.TS_ERR_INVALID
+    assert B.ts_pick_chunk_size([128], [0.01], 4, 0.0) == B.TS_ERR_INVALID
+    assert B.ts_convertible_prefill_velocity(64, 64.0, 0.1) == 0.0
+    assert B.ts_reserved_pages(0.0, 0.25, 16) == 0
