@@ -11,6 +11,13 @@ Plain restatements of the paper's counting rules, used to check the library's co
 * Sec. 4.4: chunk size bounds (prefill tokens + decode batch size) of one iteration;
   Eq. 5: V_D^{P'} = (chunk_size - batch_size) / TPOT_SLO.
 * Eq. 6: Mem_Reserved = V_D^{P'} * Mem_T * TTFT_SLO.
+* Eq. 2: prefillers needed I^P = lambda / min(V_P, V_BW); Eq. 3: decoder demand
+  I^D = sum over buckets of lambda'(b) / V_D(b); Eq. 4: regular decoders I^D_r = max(I^D - I^D_c, 0).
+  The Scaler allocates the minimum number of instances that provides the velocity (Sec. 4.3), so
+  counts are rounded up (Fig. 7: 10 tokens/s against 8 per instance -> 2).
+* Algorithm 1: a prefill task goes to the first prefiller whose estimated waiting time
+  inflight_tokens / velocity is within the request's SLO, else to the first Convertible Decoder
+  that passes the same test with its V_D^{P'}, else it is queued.
 * Sec. 4.4, chunk-size selection: the iteration time is profiled while the prefill chunk grows,
   until the TPOT SLO is violated; the chunk size chosen is the largest one before that.
 """
@@ -43,6 +50,37 @@ def convertible_prefill_velocity(chunk_size: int, batch_size: float, tpot_slo_s:
 def reserved_memory(v_dp: float, mem_per_token: float, ttft_slo_s: float) -> float:
     """Eq. 6."""
     return v_dp * mem_per_token * ttft_slo_s
+
+
+def prefiller_instances(token_rate: float, v_prefill: float, v_network: float) -> int:
+    """Eq. 2, rounded up to whole instances."""
+    return int(math.ceil(token_rate / min(v_prefill, v_network)))
+
+
+def decoder_demand(rates, velocities) -> float:
+    """Eq. 3: the (real-valued) number of decoders the per-bucket token rates ask for."""
+    total = 0.0
+    for lam, v in zip(rates, velocities):
+        total += lam / v
+    return total
+
+
+def regular_decoders(demand: float, convertible: int) -> int:
+    """Eq. 4 on whole instances."""
+    return max(int(math.ceil(demand)) - convertible, 0)
+
+
+def route_prefill(prefiller_inflight, prefiller_velocity, cd_inflight, cd_velocity, slo_s: float):
+    """Algorithm 1. Returns ("prefiller", i), ("convertible", i) or ("queue", -1)."""
+    for i, (tok, v) in enumerate(zip(prefiller_inflight, prefiller_velocity)):
+        waiting_time = tok / v
+        if waiting_time <= slo_s:
+            return "prefiller", i
+    for i, (tok, v) in enumerate(zip(cd_inflight, cd_velocity)):
+        waiting_time = tok / v
+        if waiting_time <= slo_s:
+            return "convertible", i
+    return "queue", -1
 
 
 def reserved_tokens(v_dp: float, ttft_slo_s: float) -> float:

@@ -307,6 +307,27 @@ def pin_fig7_worked_example():
         assert velocity.request_policy_fires(int(n_req), float(thr)) == bool(int(exp_fire))
 
 
+def pin_scaler_and_router():
+    """Eq. 2-4 and Algorithm 1 on hand-worked cases."""
+    # Fig. 7's numbers through Eq. 2 (network never the bottleneck): 10 tokens/s over 8 -> 2
+    assert velocity.prefiller_instances(10.0, 8.0, 1e9) == 2
+    assert velocity.prefiller_instances(10.0, 80.0, 4.0) == 3          # the smaller velocity decides
+    assert velocity.prefiller_instances(16.0, 8.0, 8.0) == 2           # exact multiples are not rounded up
+    # Eq. 3 with two buckets: 6000/4000 + 9000/12000 = 2.25 decoders; Eq. 4 with one convertible: 3 - 1
+    d = velocity.decoder_demand([6000.0, 9000.0], [4000.0, 12000.0])
+    assert abs(d - 2.25) < 1e-12
+    assert velocity.regular_decoders(d, 1) == 2 and velocity.regular_decoders(d, 5) == 0
+    # Algorithm 1: waiting times 0.5 s and 0.2 s on the prefillers, 0.1 s on the convertible decoder
+    pre_tok, pre_v = [7000.0, 2800.0], [14000.0, 14000.0]
+    cd_tok, cd_v = [2048.0], [20480.0]
+    assert velocity.route_prefill(pre_tok, pre_v, cd_tok, cd_v, 0.25) == ("prefiller", 1)    # first one within the SLO
+    assert velocity.route_prefill(pre_tok, pre_v, cd_tok, cd_v, 0.6) == ("prefiller", 0)
+    assert velocity.route_prefill(pre_tok, pre_v, cd_tok, cd_v, 0.15) == ("convertible", 0)  # second round
+    assert velocity.route_prefill(pre_tok, pre_v, cd_tok, cd_v, 0.05) == ("queue", -1)
+    assert velocity.route_prefill(pre_tok, pre_v, cd_tok, cd_v, 0.2) == ("prefiller", 1)     # the bound is inclusive
+    assert velocity.route_prefill([], [], [], [], 1.0) == ("queue", -1)
+
+
 def pin_chunk_size_selection():
     """Sec. 4.4 against a closed form: with an iteration time that is affine in the prefill
     tokens, a + b*T, the largest admissible T is floor((SLO - a) / b) on a unit grid."""
@@ -348,7 +369,7 @@ PINS = [pin_single_key_returns_its_value, pin_two_keys_logistic_weights,
         pin_table_permutation_invariance, pin_decode_equals_last_prefill_row,
         pin_chunked_equals_unchunked, pin_softmax_weights_and_convexity, pin_gqa_group_symmetry,
         pin_needle_visibility, pin_every_position_is_gathered_from_its_slot,
-        pin_append_writes_exactly_the_live_slots, pin_fig7_worked_example, pin_eq5_eq6_and_counters, pin_chunk_size_selection]
+        pin_append_writes_exactly_the_live_slots, pin_fig7_worked_example, pin_eq5_eq6_and_counters, pin_chunk_size_selection, pin_scaler_and_router]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=[p.__name__ for p in PINS])
