@@ -293,6 +293,36 @@ double ts_reserved_memory(double prefill_velocity, double mem_per_token, double 
 int32_t ts_reserved_pages(double prefill_velocity, double ttft_slo_s, int32_t page_size);
 
 /*
+ * The Token Velocity policy around the step (Sec. 4.3, Sec. 4.5.1). Host-only arithmetic fed by
+ * rates the caller measures and by velocities profiled with ts_velocity / ts_report_step_time.
+ *
+ * ts_prefiller_instances: Eq. 2, I^P = lambda / min(V_P, V_BW), as the minimum whole number of
+ * instances whose velocity covers the input token rate (rounded up). 0 for a non-positive rate,
+ * TS_ERR_INVALID (negative) for a non-positive velocity.
+ * ts_decoder_demand: Eq. 3, I^D = sum over the n_buckets request buckets of
+ * token_rate[b] / velocity[b], as a real number (the paper compares 3.2 against 3 provisioned);
+ * -1.0 for null arrays, n_buckets <= 0, a negative rate or a non-positive velocity.
+ * ts_regular_decoders: Eq. 4, I^D_r = max(ceil(I^D) - I^D_c, 0), the Convertible Decoders being a
+ * fixed pool that is never scaled.
+ *
+ * ts_route_prefill: Algorithm 1. The request goes to the first of the n_prefillers prefillers
+ * whose estimated waiting time inflight_tokens / velocity is <= slo_s; failing that to the first
+ * of the n_convertible Convertible Decoders that passes the same test with its prefill velocity
+ * V_D^{P'} (Eq. 5); failing that it is queued. *kind_out: TS_ROUTE_PREFILLER, TS_ROUTE_CONVERTIBLE
+ * or TS_ROUTE_QUEUE; returns the chosen index (0 when queued) or TS_ERR_INVALID for a null
+ * kind_out, a null array with a positive count, a negative in-flight count or a non-positive
+ * velocity. Arrays are HOST memory and only read.
+ */
+enum { TS_ROUTE_PREFILLER = 0, TS_ROUTE_CONVERTIBLE = 1, TS_ROUTE_QUEUE = 2 };
+int32_t ts_prefiller_instances(double token_rate, double prefill_velocity, double network_velocity);
+double ts_decoder_demand(const double* token_rate, const double* velocity, int32_t n_buckets);
+int32_t ts_regular_decoders(double decoder_demand, int32_t convertible_decoders);
+int32_t ts_route_prefill(const double* prefiller_inflight_tokens, const double* prefiller_velocity,
+                         int32_t n_prefillers, const double* convertible_inflight_tokens,
+                         const double* convertible_prefill_velocity, int32_t n_convertible, double slo_s,
+                         int32_t* kind_out);
+
+/*
  * ts_plan_step: host-only. Validates the step exactly as ts_mixed_step does and writes the
  * work list it would launch: one record of 8 int32 per work item
  *   {row, kind (0 decode split, 1 prefill tile), q_begin, q_count, k_begin, k_end,

@@ -68,7 +68,8 @@ EXPORTS = ["ts_pool_bytes", "ts_workspace_bytes", "ts_create", "ts_destroy", "ts
            "ts_velocity", "ts_report_step_time", "ts_prefill_budget", "ts_plan_step",
            "ts_last_device_status", "ts_last_cuda_error", "ts_strerror", "ts_profile_enable",
            "ts_profile_read", "ts_decode_attention_static", "ts_alloc_step", "ts_pick_chunk_size",
-           "ts_convertible_prefill_velocity", "ts_reserved_memory", "ts_reserved_pages"]
+           "ts_convertible_prefill_velocity", "ts_reserved_memory", "ts_reserved_pages",
+           "ts_prefiller_instances", "ts_decoder_demand", "ts_regular_decoders", "ts_route_prefill"]
 
 _lib = None
 
@@ -118,6 +119,15 @@ def lib() -> ctypes.CDLL:
         L.ts_reserved_memory.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double]
         L.ts_reserved_pages.restype = ctypes.c_int32
         L.ts_reserved_pages.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_int32]
+        dp = ctypes.POINTER(ctypes.c_double)
+        L.ts_prefiller_instances.restype = ctypes.c_int32
+        L.ts_prefiller_instances.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double]
+        L.ts_decoder_demand.restype = ctypes.c_double
+        L.ts_decoder_demand.argtypes = [dp, dp, ctypes.c_int32]
+        L.ts_regular_decoders.restype = ctypes.c_int32
+        L.ts_regular_decoders.argtypes = [ctypes.c_double, ctypes.c_int32]
+        L.ts_route_prefill.restype = ctypes.c_int32
+        L.ts_route_prefill.argtypes = [dp, dp, ctypes.c_int32, dp, dp, ctypes.c_int32, ctypes.c_double, _i32p]
         L.ts_last_device_status.argtypes = [vp, vp, _i32p]
         L.ts_last_cuda_error.argtypes = [vp]
         L.ts_profile_enable.argtypes = [vp, ctypes.c_int]
@@ -255,6 +265,39 @@ def ts_reserved_memory(prefill_velocity: float, mem_per_token: float, ttft_slo_s
 
 def ts_reserved_pages(prefill_velocity: float, ttft_slo_s: float, page_size: int = 16) -> int:
     return lib().ts_reserved_pages(prefill_velocity, ttft_slo_s, page_size)
+
+
+TS_ROUTE_PREFILLER, TS_ROUTE_CONVERTIBLE, TS_ROUTE_QUEUE = 0, 1, 2
+
+
+def _doubles(values):
+    n = len(values)
+    return (ctypes.c_double * max(n, 1))(*[float(v) for v in values]), n
+
+
+def ts_prefiller_instances(token_rate: float, prefill_velocity: float, network_velocity: float) -> int:
+    return lib().ts_prefiller_instances(token_rate, prefill_velocity, network_velocity)
+
+
+def ts_decoder_demand(token_rate, velocity) -> float:
+    a, n = _doubles(token_rate)
+    b, _ = _doubles(velocity)
+    return lib().ts_decoder_demand(a, b, n)
+
+
+def ts_regular_decoders(decoder_demand: float, convertible_decoders: int) -> int:
+    return lib().ts_regular_decoders(decoder_demand, convertible_decoders)
+
+
+def ts_route_prefill(prefiller_inflight, prefiller_velocity, convertible_inflight, convertible_velocity, slo_s: float):
+    """Returns (index or error code, kind)."""
+    pa, np_ = _doubles(prefiller_inflight)
+    pv, _ = _doubles(prefiller_velocity)
+    ca, nc = _doubles(convertible_inflight)
+    cv, _ = _doubles(convertible_velocity)
+    kind = ctypes.c_int32(-1)
+    idx = lib().ts_route_prefill(pa, pv, np_, ca, cv, nc, slo_s, ctypes.byref(kind))
+    return idx, kind.value
 
 
 def ts_plan_step(ctx, step: ts_step):

@@ -867,6 +867,56 @@ int32_t ts_reserved_pages(double prefill_velocity, double ttft_slo_s, int32_t pa
   return pages > 2147483647.0 ? 2147483647 : (int32_t)pages;
 }
 
+int32_t ts_prefiller_instances(double token_rate, double prefill_velocity, double network_velocity) {
+  if (!(prefill_velocity > 0.0) || !(network_velocity > 0.0)) return TS_ERR_INVALID;
+  if (!(token_rate > 0.0)) return 0;
+  const double n = std::ceil(token_rate / std::min(prefill_velocity, network_velocity));
+  return n > 2147483647.0 ? 2147483647 : (int32_t)n;
+}
+
+double ts_decoder_demand(const double* token_rate, const double* velocity, int32_t n_buckets) {
+  if (!token_rate || !velocity || n_buckets <= 0) return -1.0;
+  double total = 0.0;
+  for (int b = 0; b < n_buckets; ++b) {
+    if (!(token_rate[b] >= 0.0) || !(velocity[b] > 0.0)) return -1.0;
+    total += token_rate[b] / velocity[b];
+  }
+  return total;
+}
+
+int32_t ts_regular_decoders(double decoder_demand, int32_t convertible_decoders) {
+  if (!(decoder_demand > 0.0)) return 0;
+  const double need = std::ceil(decoder_demand) - (double)std::max(convertible_decoders, 0);
+  return need <= 0.0 ? 0 : need > 2147483647.0 ? 2147483647 : (int32_t)need;
+}
+
+int32_t ts_route_prefill(const double* prefiller_inflight_tokens, const double* prefiller_velocity,
+                         int32_t n_prefillers, const double* convertible_inflight_tokens,
+                         const double* convertible_prefill_velocity, int32_t n_convertible, double slo_s,
+                         int32_t* kind_out) {
+  if (!kind_out || n_prefillers < 0 || n_convertible < 0) return TS_ERR_INVALID;
+  if (n_prefillers > 0 && (!prefiller_inflight_tokens || !prefiller_velocity)) return TS_ERR_INVALID;
+  if (n_convertible > 0 && (!convertible_inflight_tokens || !convertible_prefill_velocity)) return TS_ERR_INVALID;
+  for (int i = 0; i < n_prefillers; ++i)
+    if (!(prefiller_inflight_tokens[i] >= 0.0) || !(prefiller_velocity[i] > 0.0)) return TS_ERR_INVALID;
+  for (int i = 0; i < n_convertible; ++i)
+    if (!(convertible_inflight_tokens[i] >= 0.0) || !(convertible_prefill_velocity[i] > 0.0)) return TS_ERR_INVALID;
+  for (int i = 0; i < n_prefillers; ++i) {          // first round: the prefillers, in order
+    if (prefiller_inflight_tokens[i] / prefiller_velocity[i] <= slo_s) {
+      *kind_out = TS_ROUTE_PREFILLER;
+      return i;
+    }
+  }
+  for (int i = 0; i < n_convertible; ++i) {         // second round: the Convertible Decoders
+    if (convertible_inflight_tokens[i] / convertible_prefill_velocity[i] <= slo_s) {
+      *kind_out = TS_ROUTE_CONVERTIBLE;
+      return i;
+    }
+  }
+  *kind_out = TS_ROUTE_QUEUE;
+  return 0;
+}
+
 int ts_plan_step(ts_ctx* c, const ts_step* st, int32_t* items, int32_t items_capacity,
                  int32_t* n_items_out) {
   if (!n_items_out) return TS_ERR_INVALID;

@@ -283,3 +283,31 @@ def test_convertible_decoder_configuration_matches_the_oracle():
     assert B.ts_pick_chunk_size([128], [0.01], 4, 0.0) == B.TS_ERR_INVALID
     assert B.ts_convertible_prefill_velocity(64, 64.0, 0.1) == 0.0
     assert B.ts_reserved_pages(0.0, 0.25, 16) == 0
+
+
+def test_scaler_and_router_match_the_oracle():
+    """Eq. 2-4 and Algorithm 1 through the C ABI against oracle/velocity.py on seeded cases."""
+    rng = np.random.Generator(np.random.Philox(45))
+    names = {B.TS_ROUTE_PREFILLER: "prefiller", B.TS_ROUTE_CONVERTIBLE: "convertible", B.TS_ROUTE_QUEUE: "queue"}
+    for _ in range(300):
+        lam, vp, vn = (float(x) for x in rng.uniform(1.0, 5e4, size=3))
+        assert B.ts_prefiller_instances(lam, vp, vn) == velocity.prefiller_instances(lam, vp, vn)
+        nb = int(rng.integers(1, 10))
+        rates, vels = rng.uniform(0.0, 4e4, size=nb), rng.uniform(5e3, 4e4, size=nb)
+        d = B.ts_decoder_demand(rates.tolist(), vels.tolist())
+        assert abs(d - velocity.decoder_demand(rates.tolist(), vels.tolist())) <= 1e-12 * max(d, 1.0)
+        ic = int(rng.integers(0, 4))
+        assert B.ts_regular_decoders(d, ic) == velocity.regular_decoders(d, ic)
+        n_p, n_c = int(rng.integers(0, 5)), int(rng.integers(0, 3))
+        pt, pv = rng.uniform(0, 2e4, size=n_p).tolist(), rng.uniform(5e3, 2e4, size=n_p).tolist()
+        ct, cv = rng.uniform(0, 2e4, size=n_c).tolist(), rng.uniform(5e3, 3e4, size=n_c).tolist()
+        slo = float(rng.choice([0.25, 0.4, 2.0]))                      # the paper's TTFT SLOs
+        idx, kind = B.ts_route_prefill(pt, pv, ct, cv, slo)
+        want_kind, want_idx = velocity.route_prefill(pt, pv, ct, cv, slo)
+        assert names[kind] == want_kind and idx == max(want_idx, 0)
+    assert B.ts_prefiller_instances(10.0, 8.0, 1e9) == 2               # Fig. 7
+    assert B.ts_prefiller_instances(0.0, 8.0, 8.0) == 0
+    assert B.ts_prefiller_instances(1.0, 0.0, 8.0) == B.TS_ERR_INVALID
+    assert B.ts_decoder_demand([1.0], [0.0]) == -1.0
+    assert B.ts_regular_decoders(0.0, 1) == 0
+    assert B.ts_route_prefill([1.0], [0.0], [], [], 1.0)[0] == B.TS_ERR_INVALID
