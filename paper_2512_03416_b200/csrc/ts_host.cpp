@@ -65,7 +65,7 @@ void compute_layout(const ts_config* c, Layout* L) {
   size_t off = 0;
   L->off_status = off; off += kAlign;
   L->off_table = off; off += align_up((size_t)R * c->max_pages_per_req * sizeof(int32_t));
-  L->off_meta = off; off += L->meta_bytes;
+  L->off_meta = off; off += kRing * L->meta_bytes;   // one metadata slot per step in flight
   L->off_delta = off; off += L->delta_bytes;
   L->off_part_acc = off;
   off += align_up((size_t)L->max_partials * c->n_q_heads * c->head_dim * sizeof(float));
@@ -92,6 +92,17 @@ struct RingBuf {
   bool in_flight = false;
 };
 
+// One slot of step metadata: a pinned host buffer, its device copy in the workspace, and the
+// two events that order them. The upload runs on the context's own copy stream, next to the
+// previous step's kernels instead of between them.
+struct MetaSlot {
+  void* host = nullptr;
+  cudaEvent_t copied = nullptr;     // copy stream: the slot's upload has finished
+  cudaEvent_t consumed = nullptr;   // caller's stream: the step that read the slot is done
+  bool copy_in_flight = false;
+  bool read_in_flight = false;
+};
+
 uint64_t splitmix64(uint64_t& s) {
   uint64_t z = (s += 0x9E3779B97F4A7C15ull);
   z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
@@ -112,9 +123,13 @@ struct ts_ctx {
   std::vector<int32_t> page_owner;  // -1 = free
   std::vector<int32_t> free_slots;  // stack
   ts_velocity_counters cnt;
-  RingBuf ring[kRing];
+  RingBuf ring[kRing];              // block-table deltas
   int ring_next = 0;
   size_t ring_bytes = 0;
+  MetaSlot meta[kRing];             // step metadata
+  int meta_next = 0;
+  int meta_cur = 0;                 // slot of the step being issued
+  cudaStream_t copy_stream = nullptr;
   bool cuda_ready = false;
   CUtensorMap kv_map;               // TMA view of the pool, box = K and V of one (page, head) half
   void* encode_fn = nullptr;        // cuTensorMapEncodeTiled
@@ -208,11 +223,15 @@ int ensure_cuda(ts_ctx* c, cudaStream_t stream) {
   if (!c->cfg.kv_pool || !c->cfg.workspace) return cuda_fail(c, cudaErrorInvalidDevicePointer);
   TS_CUDA(c, cudaSetDevice(c->cfg.device));
   if (!c->cuda_ready) {
-    c->ring_bytes = std::max(c->L.meta_bytes, c->L.delta_bytes);
+    c->ring_bytes = c->L.delta_bytes;
     for (int i = 0; i < kRing; ++i) {
       TS_CUDA(c, cudaHostAlloc(&c->ring[i].host, c->ring_bytes, cudaHostAllocDefault));
       TS_CUDA(c, cudaEventCreateWithFlags(&c->ring[i].ev, cudaEventDisableTiming));
+      TS_CUDA(c, cudaHostAlloc(&c->meta[i].host, c->L.meta_bytes, cudaHostAllocDefault));
+      TS_CUDA(c, cudaEventCreateWithFlags(&c->meta[i].copied, cudaEventDisableTiming));
+      TS_CUDA(c, cudaEventCreateWithFlags(&c->meta[i].consumed, cudaEventDisableTiming));
     }
+    TS_CUDA(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
     TS_CUDA(c, cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->cfg.device));
     int rc = make_kv_maps(c);
     if (rc != TS_OK) return rc;
@@ -366,11 +385,19 @@ int sync_tables(ts_ctx* c, const ts_step* st, cudaStream_t stream) {
   return TS_OK;
 }
 
+// Sends the step's metadata to the next device slot. The copy goes over the context's copy stream:
+// it only has to wait for the step that last read this slot (kRing steps ago), so it runs while
+// the previous step's kernels are still busy, and the caller's stream just waits for its event.
 int upload_meta(ts_ctx* c, const ts_step* st, int n_items, int n_combines, cudaStream_t stream) {
-  RingBuf* rb;
-  int rc = ring_acquire(c, &rb);
-  if (rc != TS_OK) return rc;
-  int32_t* m = (int32_t*)rb->host;
+  const int slot = c->meta_next;
+  c->meta_next = (c->meta_next + 1) % kRing;
+  c->meta_cur = slot;
+  MetaSlot& ms = c->meta[slot];
+  if (ms.copy_in_flight) {                 // the pinned buffer is free once its last upload is done
+    TS_CUDA(c, cudaEventSynchronize(ms.copied));
+    ms.copy_in_flight = false;
+  }
+  int32_t* m = (int32_t*)ms.host;
   const int R = st->n_rows;
   std::memcpy(m + c->L.m_row_slot, st->slot, sizeof(int32_t) * R);
   std::memcpy(m + c->L.m_row_ctx, st->ctx_len, sizeof(int32_t) * R);
@@ -385,12 +412,26 @@ int upload_meta(ts_ctx* c, const ts_step* st, int n_items, int n_combines, cudaS
     std::memcpy(m + c->L.m_combines, c->combines.data(), sizeof(CombineItem) * n_combines);
     used = c->L.m_combines + (size_t)n_combines * 4;
   }
-  return ring_send(c, rb, c->L.off_meta, used * sizeof(int32_t), stream);
+  if (ms.read_in_flight) TS_CUDA(c, cudaStreamWaitEvent(c->copy_stream, ms.consumed, 0));
+  TS_CUDA(c, cudaMemcpyAsync((char*)c->cfg.workspace + c->L.off_meta + (size_t)slot * c->L.meta_bytes, ms.host,
+                             used * sizeof(int32_t), cudaMemcpyHostToDevice, c->copy_stream));
+  TS_CUDA(c, cudaEventRecord(ms.copied, c->copy_stream));
+  ms.copy_in_flight = true;
+  TS_CUDA(c, cudaStreamWaitEvent(stream, ms.copied, 0));
+  return TS_OK;
+}
+
+// After the step's kernels: marks the slot as read once the caller's stream gets here.
+int release_meta(ts_ctx* c, cudaStream_t stream) {
+  MetaSlot& ms = c->meta[c->meta_cur];
+  TS_CUDA(c, cudaEventRecord(ms.consumed, stream));
+  ms.read_in_flight = true;
+  return TS_OK;
 }
 
 void fill_device(ts_ctx* c, const ts_step* st, int64_t n_tokens, ts::StepDevice* d) {
   char* ws = (char*)c->cfg.workspace;
-  const int32_t* meta = (const int32_t*)(ws + c->L.off_meta);
+  const int32_t* meta = (const int32_t*)(ws + c->L.off_meta + (size_t)c->meta_cur * c->L.meta_bytes);
   d->pool = (uint16_t*)c->cfg.kv_pool;
   d->table = (int32_t*)(ws + c->L.off_table);
   d->status = (int32_t*)(ws + c->L.off_status);
@@ -558,6 +599,8 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
     c->cnt.prefill_tokens += (uint64_t)n_prefill;
     c->cnt.decode_tokens += (uint64_t)n_decode;
   }
+  rc = release_meta(c, stream);
+  if (rc != TS_OK) return rc;
   if (!(st->flags & TS_STEP_KEEP_LEN)) {
     for (int r = 0; r < st->n_rows; ++r) c->slots[st->slot[r]].n_tokens += st->q_len[r];
   }
@@ -624,7 +667,13 @@ int ts_destroy(ts_ctx* c) {
       if (c->ring[i].in_flight) cudaEventSynchronize(c->ring[i].ev);
       if (c->ring[i].ev) cudaEventDestroy(c->ring[i].ev);
       if (c->ring[i].host) cudaFreeHost(c->ring[i].host);
+      if (c->meta[i].copy_in_flight) cudaEventSynchronize(c->meta[i].copied);
+      if (c->meta[i].read_in_flight) cudaEventSynchronize(c->meta[i].consumed);
+      if (c->meta[i].copied) cudaEventDestroy(c->meta[i].copied);
+      if (c->meta[i].consumed) cudaEventDestroy(c->meta[i].consumed);
+      if (c->meta[i].host) cudaFreeHost(c->meta[i].host);
     }
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   }
   for (cudaEvent_t e : c->prof_events) cudaEventDestroy(e);
   delete c;
