@@ -18,7 +18,8 @@ using ts::TableDelta;
 using ts::WorkItem;
 
 constexpr int kRing = 4;                  // pinned metadata buffers in flight
-constexpr int kDeltaCapacity = 32768;     // table entries per upload batch
+constexpr int kDeltaCapacity = 32768;     // table entries per upload batch (bulk loads)
+constexpr int kSlotDeltas = 4096;         // table entries that ride along with a step's metadata
 constexpr int kDefaultSplit = 2048;       // keys per decode split (measured: 1024..4096 equally good)
 constexpr int kDefaultMaxTokens = 16384;  // step size bound when chunk_size == 0
 constexpr size_t kAlign = 256;
@@ -29,7 +30,7 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 struct Layout {
   int max_tokens, max_partials, max_items;
   size_t off_status, off_table, off_meta, off_delta, off_part_acc, off_part_ml, off_stage;
-  size_t meta_bytes, delta_bytes, stage_q_bytes, stage_kv_bytes, total;
+  size_t meta_bytes, slot_bytes, delta_bytes, stage_q_bytes, stage_kv_bytes, total;
   // int32 offsets inside the meta area
   size_t m_row_slot, m_row_ctx, m_row_qlen, m_row_tok0, m_items, m_combines, m_end;
 };
@@ -65,7 +66,9 @@ void compute_layout(const ts_config* c, Layout* L) {
   size_t off = 0;
   L->off_status = off; off += kAlign;
   L->off_table = off; off += align_up((size_t)R * c->max_pages_per_req * sizeof(int32_t));
-  L->off_meta = off; off += kRing * L->meta_bytes;   // one metadata slot per step in flight
+  // one slot per step in flight: the step's metadata, then up to kSlotDeltas block-table entries
+  L->slot_bytes = L->meta_bytes + align_up((size_t)kSlotDeltas * sizeof(TableDelta));
+  L->off_meta = off; off += kRing * L->slot_bytes;
   L->off_delta = off; off += L->delta_bytes;
   L->off_part_acc = off;
   off += align_up((size_t)L->max_partials * c->n_q_heads * c->head_dim * sizeof(float));
@@ -227,7 +230,7 @@ int ensure_cuda(ts_ctx* c, cudaStream_t stream) {
     for (int i = 0; i < kRing; ++i) {
       TS_CUDA(c, cudaHostAlloc(&c->ring[i].host, c->ring_bytes, cudaHostAllocDefault));
       TS_CUDA(c, cudaEventCreateWithFlags(&c->ring[i].ev, cudaEventDisableTiming));
-      TS_CUDA(c, cudaHostAlloc(&c->meta[i].host, c->L.meta_bytes, cudaHostAllocDefault));
+      TS_CUDA(c, cudaHostAlloc(&c->meta[i].host, c->L.slot_bytes, cudaHostAllocDefault));
       TS_CUDA(c, cudaEventCreateWithFlags(&c->meta[i].copied, cudaEventDisableTiming));
       TS_CUDA(c, cudaEventCreateWithFlags(&c->meta[i].consumed, cudaEventDisableTiming));
     }
@@ -357,7 +360,8 @@ void plan(ts_ctx* c, const ts_step* st) {
 // Brings the device copy of the rows' block tables up to date (entries added since the last
 // step that used the slot). Entries travel by value through the pinned ring, so later host-side
 // changes cannot alter what an already enqueued step sees.
-int sync_tables(ts_ctx* c, const ts_step* st, cudaStream_t stream) {
+int sync_tables(ts_ctx* c, const ts_step* st, cudaStream_t stream, int* n_slot_deltas) {
+  *n_slot_deltas = 0;
   c->deltas.clear();
   for (int r = 0; r < st->n_rows; ++r) {
     Slot& s = c->slots[st->slot[r]];
@@ -365,6 +369,12 @@ int sync_tables(ts_ctx* c, const ts_step* st, cudaStream_t stream) {
     for (int i = s.synced_pages; i < s.n_pages; ++i)
       c->deltas.push_back(TableDelta{st->slot[r], i, row[i]});
     s.synced_pages = s.n_pages;
+  }
+  if (c->deltas.size() <= (size_t)kSlotDeltas) {
+    // the usual case (a few rows crossed a page boundary): the entries travel with the step's
+    // metadata over the copy stream, see upload_meta
+    *n_slot_deltas = (int)c->deltas.size();
+    return TS_OK;
   }
   size_t at = 0;
   while (at < c->deltas.size()) {
@@ -388,7 +398,7 @@ int sync_tables(ts_ctx* c, const ts_step* st, cudaStream_t stream) {
 // Sends the step's metadata to the next device slot. The copy goes over the context's copy stream:
 // it only has to wait for the step that last read this slot (kRing steps ago), so it runs while
 // the previous step's kernels are still busy, and the caller's stream just waits for its event.
-int upload_meta(ts_ctx* c, const ts_step* st, int n_items, int n_combines, cudaStream_t stream) {
+int upload_meta(ts_ctx* c, const ts_step* st, int n_items, int n_combines, int n_slot_deltas, cudaStream_t stream) {
   const int slot = c->meta_next;
   c->meta_next = (c->meta_next + 1) % kRing;
   c->meta_cur = slot;
@@ -412,12 +422,24 @@ int upload_meta(ts_ctx* c, const ts_step* st, int n_items, int n_combines, cudaS
     std::memcpy(m + c->L.m_combines, c->combines.data(), sizeof(CombineItem) * n_combines);
     used = c->L.m_combines + (size_t)n_combines * 4;
   }
+  char* dev_slot = (char*)c->cfg.workspace + c->L.off_meta + (size_t)slot * c->L.slot_bytes;
+  if (n_slot_deltas > 0)
+    std::memcpy((char*)ms.host + c->L.meta_bytes, c->deltas.data(), (size_t)n_slot_deltas * sizeof(TableDelta));
   if (ms.read_in_flight) TS_CUDA(c, cudaStreamWaitEvent(c->copy_stream, ms.consumed, 0));
-  TS_CUDA(c, cudaMemcpyAsync((char*)c->cfg.workspace + c->L.off_meta + (size_t)slot * c->L.meta_bytes, ms.host,
-                             used * sizeof(int32_t), cudaMemcpyHostToDevice, c->copy_stream));
+  TS_CUDA(c, cudaMemcpyAsync(dev_slot, ms.host, used * sizeof(int32_t), cudaMemcpyHostToDevice, c->copy_stream));
+  if (n_slot_deltas > 0)
+    TS_CUDA(c, cudaMemcpyAsync(dev_slot + c->L.meta_bytes, (char*)ms.host + c->L.meta_bytes,
+                               (size_t)n_slot_deltas * sizeof(TableDelta), cudaMemcpyHostToDevice, c->copy_stream));
   TS_CUDA(c, cudaEventRecord(ms.copied, c->copy_stream));
   ms.copy_in_flight = true;
   TS_CUDA(c, cudaStreamWaitEvent(stream, ms.copied, 0));
+  if (n_slot_deltas > 0) {
+    char* ws = (char*)c->cfg.workspace;
+    TS_CUDA(c, ts::launch_table_update((int32_t*)(ws + c->L.off_table), c->cfg.max_pages_per_req,
+                                       c->cfg.max_requests, (int32_t*)(ws + c->L.off_status),
+                                       (const TableDelta*)(dev_slot + c->L.meta_bytes), n_slot_deltas, stream));
+    ++c->cnt.kernel_launches;
+  }
   return TS_OK;
 }
 
@@ -431,7 +453,7 @@ int release_meta(ts_ctx* c, cudaStream_t stream) {
 
 void fill_device(ts_ctx* c, const ts_step* st, int64_t n_tokens, ts::StepDevice* d) {
   char* ws = (char*)c->cfg.workspace;
-  const int32_t* meta = (const int32_t*)(ws + c->L.off_meta + (size_t)c->meta_cur * c->L.meta_bytes);
+  const int32_t* meta = (const int32_t*)(ws + c->L.off_meta + (size_t)c->meta_cur * c->L.slot_bytes);
   d->pool = (uint16_t*)c->cfg.kv_pool;
   d->table = (int32_t*)(ws + c->L.off_table);
   d->status = (int32_t*)(ws + c->L.off_status);
@@ -513,11 +535,12 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
   if (attention) plan(c, st);
   rc = ensure_cuda(c, stream);
   if (rc != TS_OK) return rc;
-  rc = sync_tables(c, st, stream);
+  int n_slot_deltas = 0;
+  rc = sync_tables(c, st, stream, &n_slot_deltas);
   if (rc != TS_OK) return rc;
   const int n_items = attention ? (int)c->items.size() : 0;
   const int n_combines = attention ? (int)c->combines.size() : 0;
-  rc = upload_meta(c, st, n_items, n_combines, stream);
+  rc = upload_meta(c, st, n_items, n_combines, n_slot_deltas, stream);
   if (rc != TS_OK) return rc;
   ts::StepDevice d;
   fill_device(c, st, n_tokens, &d);
