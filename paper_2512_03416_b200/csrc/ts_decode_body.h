@@ -224,16 +224,27 @@ __device__ __forceinline__ void decode_units(const StepDevice& s, const CUtensor
         __syncwarp();
       }
       // ---- S^T = K Q^T : 16 keys x 8 heads per n-tile
-      float sc[NH][4];
+      // (two accumulators per n-tile, even and odd k-steps: half the dependent MMA chain)
+      float sc[NH][4], sc_odd[NH][4];
 #pragma unroll
-      for (int nh = 0; nh < NH; ++nh) sc[nh][0] = sc[nh][1] = sc[nh][2] = sc[nh][3] = 0.f;
+      for (int nh = 0; nh < NH; ++nh) {
+        sc[nh][0] = sc[nh][1] = sc[nh][2] = sc[nh][3] = 0.f;
+        sc_odd[nh][0] = sc_odd[nh][1] = sc_odd[nh][2] = sc_odd[nh][3] = 0.f;
+      }
 #pragma unroll
       for (int ks = 0; ks < D / 16; ++ks) {
         uint32_t a[4];
         const int mi = lane >> 3;
         ldsm_x4(a, sp + page_off<D>(0, (mi & 1) * 8 + (lane & 7), 2 * ks + (mi >> 1)));
 #pragma unroll
-        for (int nh = 0; nh < NH; ++nh) mma16816(sc[nh], a, qf[nh][ks][0], qf[nh][ks][1]);
+        for (int nh = 0; nh < NH; ++nh) mma16816((ks & 1) ? sc_odd[nh] : sc[nh], a, qf[nh][ks][0], qf[nh][ks][1]);
+      }
+#pragma unroll
+      for (int nh = 0; nh < NH; ++nh) {
+        sc[nh][0] += sc_odd[nh][0];
+        sc[nh][1] += sc_odd[nh][1];
+        sc[nh][2] += sc_odd[nh][2];
+        sc[nh][3] += sc_odd[nh][3];
       }
       // ---- online softmax per head (this lane: heads 2t, 2t+1 of each n-tile; keys g, g+8)
       uint32_t pb[NH][2];
