@@ -53,7 +53,7 @@ constexpr int kBlockKeys = 128;
 constexpr int kD = 128;
 constexpr int kTileBytes = 128 * kD * 2;        // one 128 x 128 bf16 operand tile: 32 KB
 constexpr int kHalfBytes = kTileBytes / 2;      // 64 head_dim columns of it
-constexpr int kKStages = 3, kVStages = 2;
+constexpr int kKStages = 2, kVStages = 3;       // measured: a third V stage is worth more than a third K stage (3%)
 constexpr float kRescaleThreshold = 8.0f;       // log2 units
 
 // shared-memory map (offsets from the 1024-aligned base)
@@ -664,7 +664,7 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
         const int g = g0 + j;
         const int st = g % stages;
         const int key0 = j * kBlockKeys;
-        if (j >= lag) announce(j - lag, lag - 1);              // K: tile j-2 (j-1 in flight); V: tile j-1
+        if (j >= lag) announce(j - lag, lag - 1);              // V: tile j-2 (j-1 in flight); K: tile j-1
         int pg_next[8];
         if (j + 1 < u.nb) fetch_pages(j + 1, pg_next);         // table loads fly while this tile is issued
         if (g >= stages) wait(empty + st, ((g / stages) & 1) ^ 1);
