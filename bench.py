@@ -323,6 +323,9 @@ def run_static(args, world, rank, local, barrier):
     ms_step = reduce_max(e0.elapsed_time(e1), world, "cuda") / K
     launches = int(lb.dec.velocity()["kernel_launches"] - v0["kernel_launches"])
     tokens = batch.n_tokens
+    status = lb.dec.device_status()                   # a bounded wait that ran out would make the timing meaningless
+    if status != 0:
+        raise SystemExit(f"the device reported status {status} during the timed steps")
 
     lb.dec.profile_enable(True)                       # separate pass: the extra events cost a little
     for _ in range(min(K, 300)):
@@ -396,6 +399,9 @@ def run_replay(args, world, rank, local, barrier):
     barrier()
     clocks = sampler.stop()
     total_ms = reduce_max(e0.elapsed_time(e1), world, "cuda")
+    status = run.dec.device_status()                  # a bounded wait that ran out would make the timing meaningless
+    if status != 0:
+        raise SystemExit(f"the device reported status {status} during the replay")
     launches = int(run.dec.velocity()["kernel_launches"])
     tokens = sum(ps.n_tokens for ps in run.steps)
     pf_tok = sum(ps.prefill_tokens for ps in run.steps)
