@@ -150,3 +150,55 @@ def test_short_bursty_replay_matches_the_oracle():
     v = run.dec.velocity()
     assert (v["steps"], v["prefill_tokens"], v["decode_tokens"], v["released_tokens"], v["released_requests"]) == \
         (mirror.steps, mirror.prefill_tokens, mirror.decode_tokens, mirror.released_tokens, mirror.released_requests)
+
+
+def test_full_size_replay_sampled_parity():
+    """The 200-step bursty replay at its full size (70B-shaped layer, up to 256 decode rows with
+    contexts up to 32768, prefill chunks up to 8192 tokens), issued exactly as the benchmark issues
+    it. The oracle mirrors every append (so the whole pool can be compared at the end) and checks
+    the attention output on a sample: steps 0, 1, every 20th and the last one, plus the first two
+    steps that carry at least 2048 prefill tokens; in a sampled step every decode row and, per
+    prefill chunk, 192 seeded tokens plus the first and last token of every 128-token stretch."""
+    trace = wl.TraceReplay()
+    run = ReplayRunner(trace, keep_host=True, nan_fill=True)
+    s = run.shape
+    n_pages, width = run.dec.cfg.n_pages, run.dec.cfg.max_pages_per_req
+    pool = np.full(s.pool_elems(n_pages), wl.BF16_NAN, np.uint16)
+    rng = np.random.default_rng(1)
+    last = len(run.steps) - 1
+    heavy = [ps.index for ps in run.steps if ps.prefill_tokens >= 2048][:2]
+    sampled = {0, 1, last} | set(range(20, last, 20)) | set(heavy)
+    checked = checked_prefill = 0
+    for ps in run.steps:
+        run.begin_step(ps)
+        for r, cached in ps.preload:
+            k, v = run.warm_ctx[r.req_id]
+            tm = _oracle_tables(run.dec, [run.slot_of[r.req_id]], width)
+            oracle.kv_append(pool, s.Hkv, s.D, s.P, tm, [0], [cached], k, v)
+        if ps.req_ids:
+            slots = ps.slots.tolist()
+            tm = _oracle_tables(run.dec, slots, width)
+            run.launch(ps)
+            q, k, v = ps.host
+            if ps.index in sampled:
+                sel, t0 = [], 0
+                for ql in ps.q_len:
+                    if ql == 1:
+                        sel.append(t0)
+                    else:
+                        edges = [t0 + e for b in range(0, ql, 128) for e in (b, min(b + 127, ql - 1))]
+                        sel.extend(edges + (t0 + rng.integers(0, ql, 192)).tolist())
+                    t0 += ql
+                sel = np.unique(np.asarray(sel, np.int32))
+                want = oracle.mixed_step(pool, s.Hq, s.Hkv, s.D, s.P, 1 / math.sqrt(s.D), tm, ps.ctx_len, ps.q_len,
+                                         q, k, v, sel=sel)
+                got = wl.bf16_bits_to_f32(from_dev(ps.out))[sel]
+                assert_parity(got, want, "paper", f"full replay step {ps.index}")
+                checked += 1
+                checked_prefill += ps.prefill_tokens > 0
+            else:
+                oracle.kv_append(pool, s.Hkv, s.D, s.P, tm, ps.ctx_len, ps.q_len, k, v)
+        run.end_step(ps)
+    assert checked >= 10 and checked_prefill >= 2
+    assert run.dec.device_status() == 0
+    assert np.array_equal(from_dev(run.dec.pool), pool), "pool differs after the full replay"
