@@ -133,3 +133,22 @@ def test_mixed_70b_shape_group8():
     got = run.step()
     assert_parity(got, want, "peaked", "70B-shaped mixed step")
     assert np.array_equal(run.pool(), pool_want)
+
+
+def test_maximum_sizes_sampled():
+    """The largest shapes the workloads allow (70B-shaped layer): a decode row whose context fills
+    a 2048-page block table (32768 tokens with its new one) and an 8192-token prefill chunk that
+    continues 24576 cached tokens, so its last token also sees 32768 keys. The oracle checks every
+    decode row and a sample of the chunk (its first and last tokens, the edges of every 128-token
+    stretch and 200 seeded tokens); the pool is compared in full."""
+    b = wl.make_batch("max", wl.LLAMA70B, [32767, 24576, 15], [1, 8192, 1], seed=31, profile="peaked",
+                      chunk_size=8194)
+    rng = np.random.default_rng(2)
+    chunk = 1 + np.unique(np.concatenate([[0, 8191], np.arange(0, 8192, 128), np.arange(127, 8192, 128),
+                                          rng.integers(0, 8192, 200)]))
+    sel = np.concatenate([[0], chunk, [8193]]).astype(np.int32)
+    want, pool_want = oracle_step(b, sel=sel)
+    run = GpuRun(b)
+    got = run.step()[sel]
+    assert_parity(got, want, "peaked", "maximum sizes")
+    assert np.array_equal(run.pool(), pool_want)
