@@ -2,7 +2,8 @@
 // and by the mixed kernel whose decode CTAs run it before they join the prefill work.
 //
 // The path is bound by HBM: every cached K/V byte is read once and used for 4*G flops.
-//   * each CTA walks a static, cost-sorted sequence of work units (decode work item x KV head);
+//   * each CTA walks a static sequence of the cost-sorted work units (decode work item x KV head),
+//     dealt forth and back over the CTAs;
 //   * K/V pages (16 tokens) arrive by TMA tensor copies, 128-byte swizzled, straight from the
 //     paged pool; the page id is a TMA coordinate, so scattered pages cost nothing extra;
 //   * every warp owns a private ring of page stages and issues its own copies: the pages of a
@@ -69,7 +70,7 @@ __device__ __forceinline__ uint32_t page_off(int kv, int r, int c) {
 }
 
 // The sequence of pages one warp works on: for unit sequence number k of this CTA
-// (unit = cta + k * n_ctas), the unit's pages j = warp, warp + W, ...
+// (unit = k * n_ctas + cta, or + n_ctas - 1 - cta for odd k), the unit's pages j = warp, warp + W, ...
 struct UnitInfo {
   int first_page, n_pg;   // pages [first_page, first_page + n_pg) of the row's block table
   int head;               // KV head
@@ -81,7 +82,9 @@ struct UnitInfo {
 
 __device__ __forceinline__ bool load_unit(const StepDevice& s, int cta, int n_ctas, int k, UnitInfo& u) {
   const int n_dec = s.n_items - s.n_prefill_items;
-  const long long unit = (long long)cta + (long long)k * n_ctas;
+  // units are sorted by length: dealing them forth and back (CTA 0 .. n-1, then n-1 .. 0) keeps the
+  // CTAs' totals close, where plain round-robin would hand CTA 0 the longest unit of every round
+  const long long unit = (long long)k * n_ctas + ((k & 1) ? (long long)(n_ctas - 1 - cta) : (long long)cta);
   if (unit >= (long long)n_dec * s.Hkv) return false;
   const WorkItem it = s.items[s.n_prefill_items + (int)(unit / s.Hkv)];
   u.head = (int)(unit % s.Hkv);
@@ -101,7 +104,7 @@ __host__ __device__ constexpr size_t decode_smem_bytes(int G) {
          (size_t)kDecWarps * STAGES * 8;
 }
 
-// Runs the decode units cta, cta + n_ctas, ... on the first kDecThreads threads of the block (the
+// Runs this CTA's share of the decode units on the first kDecThreads threads of the block (the
 // caller keeps any other threads away). `smem` is the 1024-byte-aligned shared-memory window
 // (decode_smem_bytes<D, STAGES>(G) bytes), `base` its shared-space address. The caller has
 // executed griddepcontrol.wait; the function leaves no copy in flight when it returns.
