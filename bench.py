@@ -41,7 +41,12 @@ WORKLOADS = {
     "config3": (wl.config3, "convertible-decoder burst, 8B-shaped layer (64 decode rows + one fresh 2048-token prefill chunk)"),
     "config4": (wl.config4, "chunked-prefill continuation, 8B-shaped layer (128 decode rows + 4 chunks of 512 tokens)"),
     "config5": (None, "bursty trace replay, 70B-shaped layer (200 steps, Gamma arrivals CV=4, <=256 decodes, one prefill task at a time)"),
+    "config5_chunked": (None, "the same bursty trace under a chunk size of 2304 (2048 prefill tokens + 256 decode rows): "
+                              "prompts continue over several steps, up to 4 requests' chunks share a step"),
 }
+# what the replays change in the trace simulator's defaults
+REPLAY_TRACE = {"config5": {}, "config5_chunked": {"chunk_size": 2304, "max_prefill_tasks": 4}}
+N_LAYERS_70B = 80          # layers of the model whose attention layer the replay runs (for the TTFT clock)
 
 
 def load_peaks():
@@ -201,7 +206,7 @@ def replay_heavy_batch():
 
 
 def make_static_batch(workload: str, rank: int):
-    if workload == "config5":
+    if workload in REPLAY_TRACE:
         return replay_heavy_batch()
     make = WORKLOADS[workload][0]
     return make(seed=rank_seed(make.__defaults__[0], rank))
@@ -373,13 +378,14 @@ def run_replay(args, world, rank, local, barrier):
     """config5: the 200-step bursty replay. Every step is issued once, in order (the state evolves);
     warm-up is a full untimed replay on a fresh instance."""
     import torch
-    from paper_2512_03416_b200.replay import ReplayRunner
+    from paper_2512_03416_b200.replay import ReplayRunner, ttft_report
 
     K = min(args.steps, 200)
     seed = rank_seed(5, rank)
 
     def fresh(keep_host=False):
-        return ReplayRunner(wl.TraceReplay(seed=seed, n_steps=K), seed=seed + 45, device=local, keep_host=keep_host)
+        return ReplayRunner(wl.TraceReplay(seed=seed, n_steps=K, **REPLAY_TRACE[args.workload]), seed=seed + 45,
+                            device=local, keep_host=keep_host)
 
     warm = fresh()
     warm.run(timed=False)                              # warm-up: every launch shape once
@@ -466,6 +472,12 @@ def run_replay(args, world, rank, local, barrier):
                          "max": float(np.max(step_ms)), "min": float(step_ms[order[0]])},
              "sum_t_roof_over_sum_t": float(sum(t_roof) / (sum(step_ms) * 1e-3)),
              "steps_with_prefill": int(sum(1 for ps in run.steps if ps.prefill_tokens > 0)),
+             # time to first token of the absorbed requests: on the trace's own clock (every step one
+             # tick), and with every step lasting its measured attention time x the model's layers
+             # (attention alone understates a layer, so this is a lower bound on a real TTFT)
+             "ttft": {"tick_s": run.trace.step_s, "trace_clock": ttft_report(run.trace, run.steps),
+                      "measured_attention_x_layers": ttft_report(run.trace, run.steps,
+                                                                 [m * 1e-3 * N_LAYERS_70B for m in step_ms])},
              "heavy_steps": {"count": len(heavy),
                              "frac": float(sum(t_roof[i] for i in heavy) / (sum(step_ms[i] for i in heavy) * 1e-3)) if heavy else None}}
     cfg = {"decode_rows": "<=%d per step" % max(ps.decode_tokens for ps in run.steps), "prefill_tokens": pf_tok,
@@ -491,7 +503,7 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    r = (run_replay if args.workload == "config5" else run_static)(args, world, rank, local, barrier)
+    r = (run_replay if args.workload in REPLAY_TRACE else run_static)(args, world, rank, local, barrier)
     peaks, peak_kind = load_peaks()
     roofline, step_roofline = rooflines(peaks, peak_kind, r["flops"], r["byts"], r["ms_step"], r["prof"], r["parts"],
                                         KERNEL_TRAFFIC_BYTES.get(args.workload))
@@ -499,7 +511,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = cpu_baseline_leg(r["batch"] if r["batch"] is not None else make_static_batch(args.workload, 0))
     if rank == 0:
-        shape = wl.LLAMA70B if args.workload == "config5" else wl.LLAMA8B
+        shape = wl.LLAMA70B if args.workload in REPLAY_TRACE else wl.LLAMA8B
         cfg = {"workload": args.workload, "description": WORKLOADS[args.workload][1], "n_q_heads": shape.Hq,
                "n_kv_heads": shape.Hkv, "head_dim": shape.D, "page_size": shape.P,
                "parallelism": f"replicas x{world}"}

@@ -50,6 +50,53 @@ class PreparedStep:
         return int(sum(1 for t in self.q_len if t == 1))
 
 
+def ttft_report(trace: wl.TraceReplay, steps, step_seconds=None, slos=(0.25, 0.4, 2.0)) -> dict:
+    """Time to first token of every request whose prefill the replay absorbed (Sec. 2.2: the time
+    from a request's arrival until its first output token), against TTFT SLOs (Sec. 6.1 uses
+    250, 400 and 2000 ms by prompt length).
+
+    ``steps``: the replay's steps in order (anything with ``index`` and rows of
+    (req_id, q_len, ctx_len), e.g. ReplayStep or PreparedStep with req_ids/q_len/ctx_len).
+    A request's first token exists when the step that holds the last chunk of its prompt ends.
+    Step i is issued at i * step_s of the trace's virtual clock, or when its predecessor has
+    ended if that is later, and lasts ``step_seconds[i]`` (default: step_s, the virtual clock
+    alone). TTFT = that end time - arrival: queueing (arrival until the step that takes the
+    first chunk is issued) plus the chunk steps. Requests in flight at step 0 are left out;
+    requests whose prefill the replay does not finish are counted as ``unfinished``.
+    """
+    prompt = {r.req_id: r for r in trace.requests}
+    first_chunk, last_chunk = {}, {}
+    end, ends, starts = 0.0, [], []
+    for i, st in enumerate(steps):
+        rows = st.rows if hasattr(st, "rows") else zip(st.req_ids, st.q_len, st.ctx_len)
+        start = max(i * trace.step_s, end)
+        end = start + (trace.step_s if step_seconds is None else float(step_seconds[i]))
+        starts.append(start)
+        ends.append(end)
+        for rid, ql, ctx in rows:
+            r = prompt.get(rid)
+            if r is None or ctx >= r.prompt_len:
+                continue                              # warm request or decode row
+            first_chunk.setdefault(rid, i)
+            if ctx + ql == r.prompt_len:
+                last_chunk[rid] = i
+    ttft, queue_s, chunk_steps = [], [], []
+    for rid, i in last_chunk.items():
+        r = prompt[rid]
+        ttft.append(ends[i] - r.arrival_s)
+        queue_s.append(starts[first_chunk[rid]] - r.arrival_s)
+        chunk_steps.append(i - first_chunk[rid] + 1)
+    t = np.asarray(ttft, dtype=np.float64)
+    out = {"requests": len(ttft), "unfinished": len(trace.requests) - len(ttft)}
+    if len(ttft):
+        out.update({"ttft_mean_s": float(t.mean()), "ttft_p50_s": float(np.percentile(t, 50)),
+                    "ttft_p99_s": float(np.percentile(t, 99)), "ttft_max_s": float(t.max()),
+                    "queue_mean_s": float(np.mean(queue_s)), "chunk_steps_mean": float(np.mean(chunk_steps)),
+                    "chunk_steps_max": int(max(chunk_steps)),
+                    "attainment": {f"{int(round(x * 1e3))}ms": float((t <= x).mean()) for x in slos}})
+    return out
+
+
 class ReplayRunner:
     def __init__(self, trace: wl.TraceReplay, seed: int = 50, device: int = 0, keep_host: bool = False,
                  pool_pages: Optional[int] = None, nan_fill: bool = False, decode_split_tokens: int = 0):

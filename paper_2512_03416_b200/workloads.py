@@ -290,6 +290,8 @@ class ReplayRequest:
     cached: int = 0          # tokens in the KV cache
     decoded: int = 0         # output tokens produced so far
     warm: bool = False       # in flight at step 0 (context preloaded)
+    admitted_step: int = -1      # step before which the request entered the instance
+    first_token_step: int = -1   # step that held the last chunk of its prompt (-1: not reached)
 
 
 @dataclass
@@ -313,16 +315,23 @@ class TraceReplay:
     chunk_size - decode rows, max_chunk) tokens; a request is admitted only while fewer than
     ``max_decodes`` requests are live. A finished prefill yields the first output token; the
     request then decodes output_len - 1 more tokens and is freed.
+
+    ``max_prefill_tasks`` > 1 generalises the rule: prefill tasks are served in arrival order,
+    each with what is left of the step's budget, and while budget is left and fewer than
+    ``max_prefill_tasks`` tasks are in progress the next queued request is admitted into the
+    same step. A step then carries chunks of several requests, and a prompt longer than the
+    budget continues over the following steps.
     """
 
     def __init__(self, seed: int = 5, shape: Shape = LLAMA70B, n_steps: int = 200, rate: float = 20.0,
                  cv: float = 4.0, step_s: float = 0.030, max_decodes: int = 256, warm: int = 192,
-                 max_chunk: int = 8192, chunk_size: int = 8448):
+                 max_chunk: int = 8192, chunk_size: int = 8448, max_prefill_tasks: int = 1):
         self.shape = shape
         self.n_steps = n_steps
         self.chunk_size = chunk_size
         self.max_chunk = max_chunk
         self.max_decodes = max_decodes
+        self.max_prefill_tasks = max_prefill_tasks
         self.step_s = step_s
         rng = np.random.Generator(np.random.Philox(seed))
         self.rng = rng
@@ -359,7 +368,7 @@ class TraceReplay:
         """Yield ReplayStep objects in order. Deterministic given the seed."""
         live: List[ReplayRequest] = []       # decoding
         queue: List[ReplayRequest] = []      # arrived, waiting for prefill
-        task: Optional[ReplayRequest] = None # the one prefill task in progress
+        tasks: List[ReplayRequest] = []      # prefill tasks in progress, in arrival order
         pending = list(self.requests)
         for s in range(self.n_steps):
             now = s * self.step_s
@@ -371,22 +380,34 @@ class TraceReplay:
                     preload.append((r, r.cached))      # the request objects advance as the replay runs
             while pending and pending[0].arrival_s <= now:
                 queue.append(pending.pop(0))
-            n_live = len(live) + (1 if task is not None else 0)
-            if task is None and queue and n_live < self.max_decodes:
-                task = queue.pop(0)
-                adds.append(task)
+
+            def admit():
+                if len(tasks) < self.max_prefill_tasks and queue and len(live) + len(tasks) < self.max_decodes:
+                    r = queue.pop(0)
+                    r.admitted_step = s
+                    tasks.append(r)
+                    adds.append(r)
+                    return True
+                return False
+
+            if not tasks:
+                admit()
             rows, frees = [], []
             for r in live:
                 rows.append((r.req_id, 1, r.cached))
             budget = self.chunk_size - len(live)
-            finished_prefill = None
-            if task is not None and budget > 0:
+            finished = []
+            i = 0
+            while budget > 0 and (i < len(tasks) or (i > 0 and admit())):
+                task = tasks[i]
+                i += 1
                 take = min(task.prompt_len - task.cached, budget, self.max_chunk)
                 if take > 0:
                     rows.append((task.req_id, take, task.cached))
                     task.cached += take
+                    budget -= take
                     if task.cached == task.prompt_len:
-                        finished_prefill = task
+                        finished.append(task)
             still = []
             for r in live:
                 r.cached += 1
@@ -396,13 +417,14 @@ class TraceReplay:
                 else:
                     still.append(r)
             live = still
-            if finished_prefill is not None:
-                finished_prefill.decoded = 1
-                if finished_prefill.output_len <= 1:
-                    frees.append(finished_prefill.req_id)
+            for r in finished:
+                r.decoded = 1
+                r.first_token_step = s
+                if r.output_len <= 1:
+                    frees.append(r.req_id)
                 else:
-                    live.append(finished_prefill)
-                task = None
+                    live.append(r)
+                tasks.remove(r)
             yield ReplayStep(s, adds, preload, rows, frees)
 
 

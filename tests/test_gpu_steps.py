@@ -152,22 +152,18 @@ def test_short_bursty_replay_matches_the_oracle():
         (mirror.steps, mirror.prefill_tokens, mirror.decode_tokens, mirror.released_tokens, mirror.released_requests)
 
 
-def test_full_size_replay_sampled_parity():
-    """The 200-step bursty replay at its full size (70B-shaped layer, up to 256 decode rows with
-    contexts up to 32768, prefill chunks up to 8192 tokens), issued exactly as the benchmark issues
-    it. The oracle mirrors every append (so the whole pool can be compared at the end) and checks
-    the attention output on a sample: steps 0, 1, every 20th and the last one, plus the first two
-    steps that carry at least 2048 prefill tokens; in a sampled step every decode row and, per
-    prefill chunk, 192 seeded tokens plus the first and last token of every 128-token stretch."""
-    trace = wl.TraceReplay()
+def _replay_sampled_parity(trace, extra_steps, min_prefill_checked):
+    """Runs a replay as the benchmark issues it. The oracle mirrors every append (so the whole pool
+    can be compared at the end) and checks the attention output on a sample: steps 0, 1, every 20th
+    and the last one, plus `extra_steps(run)`; in a sampled step every decode row and, per prefill
+    chunk, 192 seeded tokens plus the first and last token of every 128-token stretch."""
     run = ReplayRunner(trace, keep_host=True, nan_fill=True)
     s = run.shape
     n_pages, width = run.dec.cfg.n_pages, run.dec.cfg.max_pages_per_req
     pool = np.full(s.pool_elems(n_pages), wl.BF16_NAN, np.uint16)
     rng = np.random.default_rng(1)
     last = len(run.steps) - 1
-    heavy = [ps.index for ps in run.steps if ps.prefill_tokens >= 2048][:2]
-    sampled = {0, 1, last} | set(range(20, last, 20)) | set(heavy)
+    sampled = {0, 1, last} | set(range(20, last, 20)) | set(extra_steps(run))
     checked = checked_prefill = 0
     for ps in run.steps:
         run.begin_step(ps)
@@ -199,6 +195,31 @@ def test_full_size_replay_sampled_parity():
             else:
                 oracle.kv_append(pool, s.Hkv, s.D, s.P, tm, ps.ctx_len, ps.q_len, k, v)
         run.end_step(ps)
-    assert checked >= 10 and checked_prefill >= 2
+    assert checked >= 10 and checked_prefill >= min_prefill_checked
     assert run.dec.device_status() == 0
     assert np.array_equal(from_dev(run.dec.pool), pool), "pool differs after the full replay"
+    return run
+
+
+def test_full_size_replay_sampled_parity():
+    """The 200-step bursty replay at its full size (70B-shaped layer, up to 256 decode rows with
+    contexts up to 32768, prefill chunks up to 8192 tokens); the first two steps that carry at
+    least 2048 prefill tokens are among the sampled ones."""
+    _replay_sampled_parity(wl.TraceReplay(),
+                           lambda run: [ps.index for ps in run.steps if ps.prefill_tokens >= 2048][:2], 2)
+
+
+def test_chunked_replay_with_several_prefill_tasks_sampled_parity():
+    """The same trace under a chunk size of 2304 tokens with up to four prefill tasks in progress
+    (Sec. 4.4: chunk size = prefill tokens + decode batch): prompts continue across steps at
+    arbitrary, not page-aligned, offsets and one step carries chunks of several requests. Sampled
+    as well: the first three steps with more than one prefill row and the first three whose chunk
+    continues an earlier one."""
+    def extra(run):
+        several = [ps.index for ps in run.steps if sum(1 for t in ps.q_len if t > 1) > 1][:3]
+        cont = [ps.index for ps in run.steps if any(t > 1 and c > 0 for t, c in zip(ps.q_len, ps.ctx_len))][:3]
+        assert len(several) == 3 and len(cont) == 3
+        return several + cont
+
+    run = _replay_sampled_parity(wl.TraceReplay(chunk_size=2304, max_prefill_tasks=4), extra, 6)
+    assert max(ps.n_tokens for ps in run.steps) <= 2304
