@@ -359,8 +359,8 @@ def run_static(args, world, rank, local, barrier):
         lb.dec.mixed_step_host(lb.slots, ql, cl, hq, hk, hv, ho, keep_len=True)
     barrier()
     t0 = time.perf_counter()
-    for _ in range(Ke):
-        lb.dec.mixed_step_host(lb.slots, ql, cl, hq, hk, hv, ho, keep_len=True)
+    for _ in range(Ke):         # enqueue only: the next step's upload overlaps this step's kernels and download
+        lb.dec.mixed_step_host(lb.slots, ql, cl, hq, hk, hv, ho, keep_len=True, wait=False)
     torch.cuda.synchronize()
     e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
     e2e = {"value": aggregate_value(tokens, world, e2e_s / Ke), "unit": UNIT,
@@ -457,7 +457,7 @@ def run_replay(args, world, rank, local, barrier):
         e2e_run.begin_step(ps)
         if pin is not None:
             hq, hk, hv, ho = pin
-            e2e_run.dec.mixed_step_host(ps.slots.tolist(), ps.q_len, ps.ctx_len, hq, hk, hv, ho)
+            e2e_run.dec.mixed_step_host(ps.slots.tolist(), ps.q_len, ps.ctx_len, hq, hk, hv, ho, wait=False)
             h2d += (hq.numel() + hk.numel() + hv.numel()) * 2
             d2h += ho.numel() * 2
         e2e_run.end_step(ps)

@@ -157,8 +157,9 @@ int ts_request_set_len(ts_ctx* ctx, int32_t slot, int32_t n_tokens);
 
 /* Step flags */
 enum {
-  TS_STEP_KEEP_LEN = 1 /* do not advance the slots' cached lengths: the same step can be
-                          issued again and rewrites the same bytes (used for timing)         */
+  TS_STEP_KEEP_LEN = 1,  /* do not advance the slots' cached lengths: the same step can be
+                            issued again and rewrites the same bytes (used for timing)       */
+  TS_STEP_HOST_ASYNC = 2 /* ts_mixed_step_host only: return once everything is enqueued      */
 };
 
 /*
@@ -213,9 +214,18 @@ int ts_mixed_step(ts_ctx* ctx, const ts_step* step, void* cuda_stream);
 
 /*
  * ts_mixed_step_host: same step with q, k_new, v_new, out in HOST memory (pinned memory makes
- * the copies asynchronous). Copies the inputs into the workspace staging area, runs the step,
- * copies out back and waits for the stream: on return out is valid. N <= chunk_size required
- * (the staging area is sized by chunk_size; chunk_size must be > 0).
+ * the copies asynchronous). Copies the inputs into a staging set of the workspace on the
+ * context's own upload stream, runs the step on cuda_stream, copies out back on the context's
+ * download stream, makes cuda_stream wait for that copy, and waits for cuda_stream: on return
+ * out is valid. N <= chunk_size required (the staging sets are sized by chunk_size; chunk_size
+ * must be > 0). The paper's decoder receives its inputs from the layers before attention, on the
+ * device; this entry point serves callers and measurements that start from host memory.
+ * With TS_STEP_HOST_ASYNC the call returns once everything is enqueued. The inputs are read at
+ * any time from the call on, so they must be final when it is made and stay unchanged, and out
+ * untouched, until cuda_stream has passed this step (synchronise it or record an event after
+ * the call). Two staging sets alternate: the upload of the next step overlaps this step's
+ * kernels and download, so a sequence of such calls is bound by the slower of the two copy
+ * directions instead of by their sum. A failed call has enqueued nothing that writes out.
  */
 int ts_mixed_step_host(ts_ctx* ctx, const ts_step* step, void* cuda_stream);
 

@@ -22,6 +22,7 @@ TS_ERR_DEVICE_TIMEOUT = -7
 TS_ERR_UNSUPPORTED = -8
 TS_ERR_WORKSPACE = -9
 TS_STEP_KEEP_LEN = 1
+TS_STEP_HOST_ASYNC = 2
 TS_DEV_BAD_PAGE = 1
 TS_DEV_TIMEOUT = 2
 TS_DEV_BAD_INDEX = 4

@@ -27,10 +27,12 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+constexpr int kStageSets = 2;   // staging sets of ts_mixed_step_host: one step uploads while another runs
+
 struct Layout {
   int max_tokens, max_partials, max_items;
   size_t off_status, off_table, off_meta, off_delta, off_part_acc, off_part_ml, off_stage;
-  size_t meta_bytes, slot_bytes, delta_bytes, stage_q_bytes, stage_kv_bytes, total;
+  size_t meta_bytes, slot_bytes, delta_bytes, stage_q_bytes, stage_kv_bytes, stage_set_bytes, total;
   // int32 offsets inside the meta area
   size_t m_row_slot, m_row_ctx, m_row_qlen, m_row_tok0, m_items, m_combines, m_end;
 };
@@ -75,7 +77,8 @@ void compute_layout(const ts_config* c, Layout* L) {
   L->off_part_ml = off; off += align_up((size_t)L->max_partials * c->n_q_heads * 2 * sizeof(float));
   L->stage_q_bytes = align_up((size_t)L->max_tokens * c->n_q_heads * c->head_dim * 2);
   L->stage_kv_bytes = align_up((size_t)L->max_tokens * c->n_kv_heads * c->head_dim * 2);
-  L->off_stage = off; off += 2 * L->stage_q_bytes + 2 * L->stage_kv_bytes;
+  L->stage_set_bytes = 2 * L->stage_q_bytes + 2 * L->stage_kv_bytes;     // q, out, k_new, v_new
+  L->off_stage = off; off += kStageSets * L->stage_set_bytes;
   L->total = off;
 }
 
@@ -133,6 +136,12 @@ struct ts_ctx {
   int meta_next = 0;
   int meta_cur = 0;                 // slot of the step being issued
   cudaStream_t copy_stream = nullptr;
+  // ts_mixed_step_host: inputs go up on up_stream, results come down on down_stream, the step
+  // itself runs on the caller's stream; the events order the three per staging set
+  cudaStream_t up_stream = nullptr, down_stream = nullptr;
+  cudaEvent_t up_done[kStageSets] = {}, step_done[kStageSets] = {}, down_done[kStageSets] = {};
+  bool stage_used[kStageSets] = {};
+  uint64_t host_steps = 0;
   bool cuda_ready = false;
   CUtensorMap kv_map;               // TMA view of the pool, box = K and V of one (page, head) half
   void* encode_fn = nullptr;        // cuTensorMapEncodeTiled
@@ -697,6 +706,19 @@ int ts_destroy(ts_ctx* c) {
       if (c->meta[i].host) cudaFreeHost(c->meta[i].host);
     }
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    if (c->up_stream) {
+      cudaStreamSynchronize(c->up_stream);
+      cudaStreamDestroy(c->up_stream);
+    }
+    if (c->down_stream) {
+      cudaStreamSynchronize(c->down_stream);
+      cudaStreamDestroy(c->down_stream);
+    }
+    for (int i = 0; i < kStageSets; ++i) {
+      if (c->up_done[i]) cudaEventDestroy(c->up_done[i]);
+      if (c->step_done[i]) cudaEventDestroy(c->step_done[i]);
+      if (c->down_done[i]) cudaEventDestroy(c->down_done[i]);
+    }
   }
   for (cudaEvent_t e : c->prof_events) cudaEventDestroy(e);
   delete c;
@@ -831,16 +853,34 @@ int ts_mixed_step_host(ts_ctx* c, const ts_step* st, void* cuda_stream) {
   if (!c->cfg.workspace) return cuda_fail(c, cudaErrorInvalidDevicePointer);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   TS_CUDA(c, cudaSetDevice(c->cfg.device));
-  char* ws = (char*)c->cfg.workspace + c->L.off_stage;
+  if (!c->up_stream) {
+    TS_CUDA(c, cudaStreamCreateWithFlags(&c->up_stream, cudaStreamNonBlocking));
+    TS_CUDA(c, cudaStreamCreateWithFlags(&c->down_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < kStageSets; ++i) {
+      TS_CUDA(c, cudaEventCreateWithFlags(&c->up_done[i], cudaEventDisableTiming));
+      TS_CUDA(c, cudaEventCreateWithFlags(&c->step_done[i], cudaEventDisableTiming));
+      TS_CUDA(c, cudaEventCreateWithFlags(&c->down_done[i], cudaEventDisableTiming));
+    }
+  }
+  // The staging sets alternate. Upload: once the set's previous result has gone down (its
+  // step is then done with the inputs too). Step: on the caller's stream, after the upload.
+  // Download: after the step. The caller's stream then waits for the download, so whatever it
+  // runs next, or a synchronisation of it, finds `out` complete; the next call's upload does
+  // not wait for any of this and overlaps this step's kernels and download.
+  const int b = (int)(c->host_steps % kStageSets);
+  char* ws = (char*)c->cfg.workspace + c->L.off_stage + (size_t)b * c->L.stage_set_bytes;
   void* dq = ws;
   void* dout = ws + c->L.stage_q_bytes;
   void* dk = ws + 2 * c->L.stage_q_bytes;
   void* dv = ws + 2 * c->L.stage_q_bytes + c->L.stage_kv_bytes;
   const size_t qb = (size_t)n * c->cfg.n_q_heads * c->cfg.head_dim * 2;
   const size_t kb = (size_t)n * c->cfg.n_kv_heads * c->cfg.head_dim * 2;
-  TS_CUDA(c, cudaMemcpyAsync(dq, st->q, qb, cudaMemcpyHostToDevice, stream));
-  TS_CUDA(c, cudaMemcpyAsync(dk, st->k_new, kb, cudaMemcpyHostToDevice, stream));
-  TS_CUDA(c, cudaMemcpyAsync(dv, st->v_new, kb, cudaMemcpyHostToDevice, stream));
+  if (c->stage_used[b]) TS_CUDA(c, cudaStreamWaitEvent(c->up_stream, c->down_done[b], 0));
+  TS_CUDA(c, cudaMemcpyAsync(dq, st->q, qb, cudaMemcpyHostToDevice, c->up_stream));
+  TS_CUDA(c, cudaMemcpyAsync(dk, st->k_new, kb, cudaMemcpyHostToDevice, c->up_stream));
+  TS_CUDA(c, cudaMemcpyAsync(dv, st->v_new, kb, cudaMemcpyHostToDevice, c->up_stream));
+  TS_CUDA(c, cudaEventRecord(c->up_done[b], c->up_stream));
+  TS_CUDA(c, cudaStreamWaitEvent(stream, c->up_done[b], 0));
   ts_step dev = *st;
   dev.q = dq;
   dev.k_new = dk;
@@ -848,11 +888,17 @@ int ts_mixed_step_host(ts_ctx* c, const ts_step* st, void* cuda_stream) {
   dev.out = dout;
   const int rc = run_step(c, &dev, cuda_stream, true);
   if (rc != TS_OK) {
-    cudaStreamSynchronize(stream);  // the input copies may still be reading the caller's buffers
+    cudaStreamSynchronize(c->up_stream);  // the input copies may still be reading the caller's buffers
     return rc;
   }
-  TS_CUDA(c, cudaMemcpyAsync(st->out, dout, qb, cudaMemcpyDeviceToHost, stream));
-  TS_CUDA(c, cudaStreamSynchronize(stream));
+  TS_CUDA(c, cudaEventRecord(c->step_done[b], stream));
+  TS_CUDA(c, cudaStreamWaitEvent(c->down_stream, c->step_done[b], 0));
+  TS_CUDA(c, cudaMemcpyAsync(st->out, dout, qb, cudaMemcpyDeviceToHost, c->down_stream));
+  TS_CUDA(c, cudaEventRecord(c->down_done[b], c->down_stream));
+  TS_CUDA(c, cudaStreamWaitEvent(stream, c->down_done[b], 0));
+  c->stage_used[b] = true;
+  ++c->host_steps;
+  if (!(st->flags & TS_STEP_HOST_ASYNC)) TS_CUDA(c, cudaStreamSynchronize(stream));
   return TS_OK;
 }
 

@@ -96,9 +96,9 @@ class Decoder:
         return torch.cuda.current_stream(self.device).cuda_stream
 
     def make_step(self, slots, q_len, ctx_len, q=None, k_new=None, v_new=None, out=None,
-                  keep_len: bool = False):
+                  keep_len: bool = False, flags: int = 0):
         return B.make_step(slots, q_len, ctx_len, _addr(q), _addr(k_new), _addr(v_new), _addr(out),
-                           B.TS_STEP_KEEP_LEN if keep_len else 0)
+                           (B.TS_STEP_KEEP_LEN if keep_len else 0) | flags)
 
     def kv_append(self, slots, q_len, ctx_len, k_new, v_new, keep_len: bool = False) -> None:
         st, _keep = self.make_step(slots, q_len, ctx_len, None, k_new, v_new, None, keep_len)
@@ -112,9 +112,13 @@ class Decoder:
         """Issue a step marshalled earlier with make_step (keeps the per-call host cost low)."""
         _check(B.ts_mixed_step(self.ctx, st, self._stream()), "ts_mixed_step")
 
-    def mixed_step_host(self, slots, q_len, ctx_len, q, k_new, v_new, out, keep_len: bool = False) -> None:
-        """q, k_new, v_new, out are HOST tensors (pinned for asynchronous copies)."""
-        st, _keep = self.make_step(slots, q_len, ctx_len, q, k_new, v_new, out, keep_len)
+    def mixed_step_host(self, slots, q_len, ctx_len, q, k_new, v_new, out, keep_len: bool = False,
+                        wait: bool = True) -> None:
+        """q, k_new, v_new, out are HOST tensors (pinned for asynchronous copies). With
+        wait=False the call only enqueues (TS_STEP_HOST_ASYNC): out is valid once the current
+        stream has passed the step, and consecutive calls overlap their copies."""
+        st, _keep = self.make_step(slots, q_len, ctx_len, q, k_new, v_new, out, keep_len,
+                                   0 if wait else B.TS_STEP_HOST_ASYNC)
         _check(B.ts_mixed_step_host(self.ctx, st, self._stream()), "ts_mixed_step_host")
 
     def step_np(self, slots, q_len, ctx_len, q, k_new, v_new, out, alloc: bool = True) -> None:

@@ -97,6 +97,58 @@ def test_repeated_step_and_host_buffers_agree():
     assert lb.dec.device_status() == 0
 
 
+def test_pipelined_host_steps_match_device_steps():
+    """Seven consecutive steps issued from pinned host buffers without waiting in between (the
+    upload of a step overlaps the previous step's kernels and download; both staging sets are
+    reused three times) give bit for bit the outputs and the pool of the same steps issued from
+    device buffers on a second decoder with the same allocator seed."""
+    s = wl.LLAMA8B
+    bank = wl.ValueBank(31, 1.0, 20)
+    mk = lambda: Decoder(s.Hq, s.Hkv, s.D, 120, 4, 64, chunk_size=400, alloc_shuffle_seed=5, nan_fill=True)
+    host, dev = mk(), mk()
+    plan = [(130, 1), (77, 1), (126, 1), (1, 1), (1, 1), (1, 1), (1, 1)]      # (new tokens of a, of b) per step
+    sa, sb = host.request_add(1, 333, 8), host.request_add(2, 90, 8)
+    assert (dev.request_add(1, 333, 8), dev.request_add(2, 90, 8)) == (sa, sb)
+    ck, cv = (bank.take(90 * s.Hkv * s.D).reshape(90, s.Hkv, s.D) for _ in range(2))
+    for d in (host, dev):
+        d.alloc_pages(sb, 90)
+        d.kv_append([sb], [90], [0], to_dev(ck), to_dev(cv))
+    len_a, len_b = 0, 90
+    pinned, dev_out = [], []
+    for qa, qb in plan:
+        n = qa + qb
+        q = bank.take(n * s.Hq * s.D).reshape(n, s.Hq, s.D)
+        k = bank.take(n * s.Hkv * s.D).reshape(n, s.Hkv, s.D)
+        v = bank.take(n * s.Hkv * s.D).reshape(n, s.Hkv, s.D)
+        bufs = [torch.from_numpy(x.view(np.int16).copy()).pin_memory() for x in (q, k, v)]
+        bufs.append(torch.full((n, s.Hq, s.D), 0x7FC0, dtype=torch.int16).pin_memory())
+        pinned.append(bufs)                                  # inputs and outputs stay alive and untouched
+        for d in (host, dev):
+            d.alloc_pages(sa, len_a + qa, for_prefill=qa > 1)
+            d.alloc_pages(sb, len_b + qb)
+        host.mixed_step_host([sa, sb], [qa, qb], [len_a, len_b], *bufs, wait=False)
+        out = torch.full((n, s.Hq, s.D), 0x7FC0, dtype=torch.int16, device="cuda")
+        dev.mixed_step([sa, sb], [qa, qb], [len_a, len_b], to_dev(q), to_dev(k), to_dev(v), out)
+        dev_out.append(out)
+        len_a += qa
+        len_b += qb
+    torch.cuda.synchronize()
+    for i, (bufs, out) in enumerate(zip(pinned, dev_out)):
+        assert np.array_equal(bufs[3].numpy(), out.cpu().numpy()), f"step {i}"
+        assert not np.any(bufs[3].numpy() == 0x7FC0)
+    assert np.array_equal(from_dev(host.pool), from_dev(dev.pool))
+    assert host.device_status() == 0 and dev.device_status() == 0
+    # a waiting call after the pipelined ones still returns with its result in place
+    q, k, v, o = pinned[-1]
+    o.fill_(0)
+    host.alloc_pages(sa, len_a + 1)
+    host.alloc_pages(sb, len_b + 1)
+    host.mixed_step_host([sa, sb], [1, 1], [len_a, len_b], q, k, v, o)
+    assert np.any(o.numpy() != 0)
+    host.close()
+    dev.close()
+
+
 def test_step_over_budget_is_refused_on_the_host():
     b = wl.make_batch("bud", wl.TINY, [10], [40], seed=5, chunk_size=32)
     lb = LoadedBatch(b)
