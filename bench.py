@@ -361,6 +361,7 @@ def run_static(args, world, rank, local, barrier):
     t0 = time.perf_counter()
     for _ in range(Ke):         # enqueue only: the next step's upload overlaps this step's kernels and download
         lb.dec.mixed_step_host(lb.slots, ql, cl, hq, hk, hv, ho, keep_len=True, wait=False)
+    lb.dec.host_fence()
     torch.cuda.synchronize()
     e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
     e2e = {"value": aggregate_value(tokens, world, e2e_s / Ke), "unit": UNIT,
@@ -461,6 +462,7 @@ def run_replay(args, world, rank, local, barrier):
             h2d += (hq.numel() + hk.numel() + hv.numel()) * 2
             d2h += ho.numel() * 2
         e2e_run.end_step(ps)
+    e2e_run.dec.host_fence()
     torch.cuda.synchronize()
     e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
     e2e_run.dec.close()

@@ -220,14 +220,23 @@ int ts_mixed_step(ts_ctx* ctx, const ts_step* step, void* cuda_stream);
  * out is valid. N <= chunk_size required (the staging sets are sized by chunk_size; chunk_size
  * must be > 0). The paper's decoder receives its inputs from the layers before attention, on the
  * device; this entry point serves callers and measurements that start from host memory.
- * With TS_STEP_HOST_ASYNC the call returns once everything is enqueued. The inputs are read at
- * any time from the call on, so they must be final when it is made and stay unchanged, and out
- * untouched, until cuda_stream has passed this step (synchronise it or record an event after
- * the call). Two staging sets alternate: the upload of the next step overlaps this step's
- * kernels and download, so a sequence of such calls is bound by the slower of the two copy
- * directions instead of by their sum. A failed call has enqueued nothing that writes out.
+ * With TS_STEP_HOST_ASYNC the call returns once everything is enqueued and cuda_stream does not
+ * wait for the download either. The inputs are read at any time from the call on, so they must
+ * be final when it is made and stay unchanged, and out untouched, until cuda_stream has passed
+ * a ts_host_fence issued after the call (then synchronise the stream or record an event), or
+ * until a later ts_mixed_step_host without the flag has returned. Three staging sets take
+ * turns: the uploads and kernels of the following steps overlap this step's download, so a
+ * sequence of such calls is bound by the slowest of upload, kernels and download instead of by
+ * their sum. A failed call has enqueued nothing that writes out.
  */
 int ts_mixed_step_host(ts_ctx* ctx, const ts_step* step, void* cuda_stream);
+
+/*
+ * ts_host_fence (the paper has no counterpart): makes cuda_stream wait, on the device, for the
+ * downloads of every ts_mixed_step_host call issued so far; the call itself does not block.
+ * TS_OK when no host step has been issued.
+ */
+int ts_host_fence(ts_ctx* ctx, void* cuda_stream);
 
 /*
  * Token Velocity counters (Sec. 3.2). Cumulative since ts_create; a monitor divides deltas by

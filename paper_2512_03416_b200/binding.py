@@ -65,7 +65,7 @@ class ts_profile(ctypes.Structure):
 
 EXPORTS = ["ts_pool_bytes", "ts_workspace_bytes", "ts_create", "ts_destroy", "ts_request_add",
            "ts_alloc_pages", "ts_block_table", "ts_block_table_set", "ts_request_free",
-           "ts_request_set_len", "ts_kv_append", "ts_mixed_step", "ts_mixed_step_host",
+           "ts_request_set_len", "ts_kv_append", "ts_mixed_step", "ts_mixed_step_host", "ts_host_fence",
            "ts_velocity", "ts_report_step_time", "ts_prefill_budget", "ts_plan_step",
            "ts_last_device_status", "ts_last_cuda_error", "ts_strerror", "ts_profile_enable",
            "ts_profile_read", "ts_decode_attention_static", "ts_alloc_step", "ts_pick_chunk_size",
@@ -106,6 +106,7 @@ def lib() -> ctypes.CDLL:
         L.ts_kv_append.argtypes = [vp, stepp, vp]
         L.ts_mixed_step.argtypes = [vp, stepp, vp]
         L.ts_mixed_step_host.argtypes = [vp, stepp, vp]
+        L.ts_host_fence.argtypes = [vp, vp]
         L.ts_velocity.argtypes = [vp, ctypes.POINTER(ts_velocity_counters)]
         L.ts_report_step_time.argtypes = [vp, ctypes.c_double]
         L.ts_prefill_budget.restype = ctypes.c_int32
@@ -232,6 +233,10 @@ def ts_mixed_step(ctx, step: ts_step, cuda_stream: int = 0) -> int:
 
 def ts_mixed_step_host(ctx, step: ts_step, cuda_stream: int = 0) -> int:
     return lib().ts_mixed_step_host(ctx, ctypes.byref(step), ctypes.c_void_p(cuda_stream))
+
+
+def ts_host_fence(ctx, cuda_stream: int = 0) -> int:
+    return lib().ts_host_fence(ctx, ctypes.c_void_p(cuda_stream))
 
 
 def ts_velocity(ctx):

@@ -27,7 +27,8 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-constexpr int kStageSets = 2;   // staging sets of ts_mixed_step_host: one step uploads while another runs
+constexpr int kStageSets = 3;   // staging sets of ts_mixed_step_host: one step uploads while another runs
+                                // and a third one's result goes down
 
 struct Layout {
   int max_tokens, max_partials, max_items;
@@ -862,11 +863,12 @@ int ts_mixed_step_host(ts_ctx* c, const ts_step* st, void* cuda_stream) {
       TS_CUDA(c, cudaEventCreateWithFlags(&c->down_done[i], cudaEventDisableTiming));
     }
   }
-  // The staging sets alternate. Upload: once the set's previous result has gone down (its
+  // The staging sets take turns. Upload: once the set's previous result has gone down (its
   // step is then done with the inputs too). Step: on the caller's stream, after the upload.
-  // Download: after the step. The caller's stream then waits for the download, so whatever it
-  // runs next, or a synchronisation of it, finds `out` complete; the next call's upload does
-  // not wait for any of this and overlaps this step's kernels and download.
+  // Download: after the step. Without TS_STEP_HOST_ASYNC the caller's stream then waits for the
+  // downloads and the call for the stream; with it nothing waits, so the following calls'
+  // uploads and kernels overlap this step's download, and ts_host_fence orders the stream
+  // behind the downloads when the caller wants the results.
   const int b = (int)(c->host_steps % kStageSets);
   char* ws = (char*)c->cfg.workspace + c->L.off_stage + (size_t)b * c->L.stage_set_bytes;
   void* dq = ws;
@@ -895,10 +897,22 @@ int ts_mixed_step_host(ts_ctx* c, const ts_step* st, void* cuda_stream) {
   TS_CUDA(c, cudaStreamWaitEvent(c->down_stream, c->step_done[b], 0));
   TS_CUDA(c, cudaMemcpyAsync(st->out, dout, qb, cudaMemcpyDeviceToHost, c->down_stream));
   TS_CUDA(c, cudaEventRecord(c->down_done[b], c->down_stream));
-  TS_CUDA(c, cudaStreamWaitEvent(stream, c->down_done[b], 0));
   c->stage_used[b] = true;
   ++c->host_steps;
-  if (!(st->flags & TS_STEP_HOST_ASYNC)) TS_CUDA(c, cudaStreamSynchronize(stream));
+  if (!(st->flags & TS_STEP_HOST_ASYNC)) {
+    const int rc2 = ts_host_fence(c, cuda_stream);
+    if (rc2 != TS_OK) return rc2;
+    TS_CUDA(c, cudaStreamSynchronize(stream));
+  }
+  return TS_OK;
+}
+
+int ts_host_fence(ts_ctx* c, void* cuda_stream) {
+  if (!c) return TS_ERR_INVALID;
+  if (!c->up_stream) return TS_OK;            // no host step has been issued
+  TS_CUDA(c, cudaSetDevice(c->cfg.device));
+  for (int i = 0; i < kStageSets; ++i)
+    if (c->stage_used[i]) TS_CUDA(c, cudaStreamWaitEvent((cudaStream_t)cuda_stream, c->down_done[i], 0));
   return TS_OK;
 }
 

@@ -115,11 +115,16 @@ class Decoder:
     def mixed_step_host(self, slots, q_len, ctx_len, q, k_new, v_new, out, keep_len: bool = False,
                         wait: bool = True) -> None:
         """q, k_new, v_new, out are HOST tensors (pinned for asynchronous copies). With
-        wait=False the call only enqueues (TS_STEP_HOST_ASYNC): out is valid once the current
-        stream has passed the step, and consecutive calls overlap their copies."""
+        wait=False the call only enqueues (TS_STEP_HOST_ASYNC): consecutive calls overlap their
+        copies and kernels, and out is valid once the current stream has passed a later
+        host_fence()."""
         st, _keep = self.make_step(slots, q_len, ctx_len, q, k_new, v_new, out, keep_len,
                                    0 if wait else B.TS_STEP_HOST_ASYNC)
         _check(B.ts_mixed_step_host(self.ctx, st, self._stream()), "ts_mixed_step_host")
+
+    def host_fence(self) -> None:
+        """Order the current stream behind the downloads of all host steps issued so far."""
+        _check(B.ts_host_fence(self.ctx, self._stream()), "ts_host_fence")
 
     def step_np(self, slots, q_len, ctx_len, q, k_new, v_new, out, alloc: bool = True) -> None:
         """One iteration from numpy int32 row arrays: grow the tables (ts_alloc_step), then

@@ -99,8 +99,7 @@ def test_repeated_step_and_host_buffers_agree():
 
 def test_pipelined_host_steps_match_device_steps():
     """Seven consecutive steps issued from pinned host buffers without waiting in between (the
-    upload of a step overlaps the previous step's kernels and download; both staging sets are
-    reused three times) give bit for bit the outputs and the pool of the same steps issued from
+    uploads and kernels of later steps overlap a step's download; every staging set is reused) give bit for bit the outputs and the pool of the same steps issued from
     device buffers on a second decoder with the same allocator seed."""
     s = wl.LLAMA8B
     bank = wl.ValueBank(31, 1.0, 20)
@@ -132,6 +131,7 @@ def test_pipelined_host_steps_match_device_steps():
         dev_out.append(out)
         len_a += qa
         len_b += qb
+    host.host_fence()
     torch.cuda.synchronize()
     for i, (bufs, out) in enumerate(zip(pinned, dev_out)):
         assert np.array_equal(bufs[3].numpy(), out.cpu().numpy()), f"step {i}"
