@@ -501,36 +501,53 @@ bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 // B200: next to streaming decode CTAs a prefill work unit costs ~3.4 us per 128-key block pair
 // plus ~3 us; the decode rows move their K/V at a fraction of the full-chip rate that falls off as
 // fewer SMs pull on HBM, faster with eight query heads per KV head (twice the arithmetic per page)
-// than with four. Measured (SMs -> fraction, linear in between):
-//   G <= 4:  48 0.53,  64 0.69, 74 0.795, 84 0.855, 100 0.905, 120 0.955, 148 1
-//   G >  4:  48 0.475, 64 0.62, 74 0.715, 84 0.78,  100 0.85,  116 0.92, 132 0.95, 148 1
+// than with four.
+//   G <= 4: an SM streams a decode unit at 70 GB/s plus ~2 us per unit, and all of them together
+//           at no more than 6.1 TB/s; the step time is flat over a range of splits, of which the
+//           middle is taken (its ends are the sensitive ones).
+//   G >  4: measured fraction of the full-chip rate by SM count, linear in between:
+//           48 0.475, 64 0.62, 74 0.715, 84 0.78, 100 0.85, 116 0.92, 132 0.95, 148 1
 int choose_prefill_ctas(const ts_ctx* c, int n_ctas, double prefill_block_pairs, double prefill_units,
-                        double decode_bytes) {
-  static const double kSm4[] = {0, 48, 64, 74, 84, 100, 120, 148};
-  static const double kRate4[] = {0, 0.53, 0.69, 0.795, 0.855, 0.905, 0.955, 1.0};
+                        double decode_bytes, double decode_units) {
   static const double kSm8[] = {0, 48, 64, 74, 84, 100, 116, 132, 148};
   static const double kRate8[] = {0, 0.475, 0.62, 0.715, 0.78, 0.85, 0.92, 0.95, 1.0};
   const bool wide = c->G > 4;
-  const double* kSm = wide ? kSm8 : kSm4;
-  const double* kRate = wide ? kRate8 : kRate4;
-  const int last = wide ? 8 : 7;
   const double w_pf = prefill_block_pairs * 3.4 + prefill_units * 3.0;
   const double t_dec_full = decode_bytes / 6.1e6;   // us at 6.1 TB/s
+  const double unit_bytes = decode_bytes / std::max(1.0, decode_units);
+  const double sm_rate = unit_bytes / (unit_bytes / 70e3 + 2.0);   // bytes per us and SM
+  auto step_time = [&](int p) {
+    double td;
+    if (wide) {
+      const double d = (double)(n_ctas - p) * 148.0 / c->n_sms;
+      int i = 1;
+      while (i < 8 && kSm8[i] < d) ++i;
+      const double rate =
+          d >= 148.0 ? 1.0 : kRate8[i - 1] + (kRate8[i] - kRate8[i - 1]) * (d - kSm8[i - 1]) / (kSm8[i] - kSm8[i - 1]);
+      td = t_dec_full / rate;
+    } else {
+      td = std::max(t_dec_full, decode_bytes / ((double)(n_ctas - p) * sm_rate));
+    }
+    return std::max(td, (w_pf + (double)(n_ctas - p) * td) / n_ctas);
+  };
   int best = 0;
   double best_t = 1e30;
   for (int p = 0; p < n_ctas; p += 2) {
-    const double d = (double)(n_ctas - p) * 148.0 / c->n_sms;
-    int i = 1;
-    while (i < last && kSm[i] < d) ++i;
-    const double rate = d >= 148.0 ? 1.0 : kRate[i - 1] + (kRate[i] - kRate[i - 1]) * (d - kSm[i - 1]) / (kSm[i] - kSm[i - 1]);
-    const double td = t_dec_full / rate;
-    const double t = std::max(td, (w_pf + (double)(n_ctas - p) * td) / n_ctas);
+    const double t = step_time(p);
     if (t < best_t - 1e-9) {
       best_t = t;
       best = p;
     }
   }
-  return best;
+  if (wide) return best;
+  int lo = -1, hi = best;
+  for (int p = 0; p < n_ctas; p += 2) {
+    if (step_time(p) <= best_t * 1.002) {
+      if (lo < 0) lo = p;
+      hi = p;
+    }
+  }
+  return ((lo + hi) / 2) & ~1;
 }
 
 int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
@@ -601,7 +618,7 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
             for (int i = c->n_prefill_items; i < n_items; ++i)
               bytes += (double)(c->items[i].k_end - c->items[i].k_begin);
             bytes *= 2.0 * c->cfg.n_kv_heads * c->cfg.head_dim * 2.0;
-            p = choose_prefill_ctas(c, n_ctas, pairs * c->cfg.n_kv_heads, (double)pf_units, bytes);
+            p = choose_prefill_ctas(c, n_ctas, pairs * c->cfg.n_kv_heads, (double)pf_units, bytes, (double)dec_units);
           }
           p = (int)std::min<long long>(p, pf_units);
           p = std::min(p, n_ctas - 1);                         // at least one CTA runs the decode splits
