@@ -364,6 +364,8 @@ def run_static(args, world, rank, local, barrier):
     lb.dec.host_fence()
     torch.cuda.synchronize()
     e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
+    if lb.dec.device_status() != 0:
+        raise SystemExit("the device reported a failure during the end-to-end loop")
     e2e = {"value": aggregate_value(tokens, world, e2e_s / Ke), "unit": UNIT,
            "h2d_bytes_per_step": int(hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2),
            "d2h_bytes_per_step": int(ho.numel() * 2), "steps": Ke, "ms_per_step": e2e_s / Ke * 1e3}
@@ -465,6 +467,8 @@ def run_replay(args, world, rank, local, barrier):
     e2e_run.dec.host_fence()
     torch.cuda.synchronize()
     e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
+    if e2e_run.dec.device_status() != 0:
+        raise SystemExit("the device reported a failure during the end-to-end replay")
     e2e_run.dec.close()
     e2e = {"value": aggregate_value(tokens, world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": int(h2d / K),
            "d2h_bytes_per_step": int(d2h / K), "steps": K, "ms_per_step": e2e_s / K * 1e3}
