@@ -181,6 +181,7 @@ __device__ __forceinline__ void decode_units(const StepDevice& s, const CUtensor
   for (int ck = 0; load_unit(s, cta, n_ctas, ck, cu); ++ck) {
     const int tok = s.row_tok0[cu.row];
     const int n = cu.k_end;   // keys at positions >= n are not visible (decode: ctx + 1 or split end)
+    const int new_pos = s.row_ctx[cu.row];   // position of the row's new token
     // Q^T fragments: lane (g, t) holds head g (and g + 8), head_dim pairs 2t, 2t+1 (+8)
     uint32_t qf[NH][D / 16][2];
 #pragma unroll
@@ -213,6 +214,23 @@ __device__ __forceinline__ void decode_units(const StepDevice& s, const CUtensor
         dead = true;
       }
       const int pos0 = cu.k_begin + j * kPageSize;   // position of the page's first slot
+      if (s.append_in_decode && new_pos >= pos0 && new_pos < pos0 + kPageSize) {
+        // KV append (Sec. 2.1) without a launch of its own: this page holds the row's new token,
+        // which is not in the pool yet. Lay its K and V over the page image in shared memory and
+        // write them to the pool page; a lane moves one 16-byte chunk of K or V.
+        constexpr int CH = D / 8;
+        const int r = new_pos - pos0;
+        const int page = cu.table_row[cu.first_page + j];
+        unsigned char* pg = smem + (sp - base);
+        for (int i = lane; i < 2 * CH; i += 32) {
+          const int kv = i / CH, c = i % CH;
+          const uint4 val = *reinterpret_cast<const uint4*>((kv ? s.v_new : s.k_new) + ((size_t)tok * s.Hkv + cu.head) * D + c * 8);
+          *reinterpret_cast<uint4*>(pg + page_off<D>(kv, r, c)) = val;
+          if ((unsigned)page < (unsigned)s.n_pages)
+            *reinterpret_cast<uint4*>(s.pool + ((((size_t)page * 2 + kv) * s.Hkv + cu.head) * kPageSize + r) * D + c * 8) = val;
+        }
+        __syncwarp();
+      }
       const bool ragged = pos0 + kPageSize > n;
       if (ragged) {
         // slots past the last token hold whatever was there before: clear their V rows so

@@ -492,6 +492,7 @@ void fill_device(ts_ctx* c, const ts_step* st, int64_t n_tokens, ts::StepDevice*
   d->max_pages_per_req = c->cfg.max_pages_per_req;
   d->max_requests = c->cfg.max_requests;
   d->scale_log2 = c->scale * 1.4426950408889634f;
+  d->append_in_decode = 0;
 }
 
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
@@ -589,7 +590,10 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
   }
   // head_dim 128 steps with prefill tiles: the mixed kernel appends the new K/V itself
   const bool append_in_kernel = attention && c->n_prefill_items > 0 && c->cfg.head_dim == 128;
-  if (!append_in_kernel) {
+  // decode-only steps: the unit that reads a row's last page writes the row's new token into it
+  const bool append_in_decode = attention && c->n_prefill_items == 0 && n_items > 0;
+  d.append_in_decode = append_in_decode;
+  if (!append_in_kernel && !append_in_decode) {
     TS_CUDA(c, ts::launch_kv_append(d, stream));
     ++c->cnt.kernel_launches;
   }

@@ -71,6 +71,7 @@ struct StepDevice {
   // shape
   int32_t n_rows, n_tokens, n_items, n_combines;
   int32_t n_prefill_items;  // items[0, n_prefill_items) are prefill tiles, the rest decode splits
+  int32_t append_in_decode; // != 0: the decode units append their rows' new K/V themselves
   int32_t Hq, Hkv, D, n_pages, max_pages_per_req, max_requests;
   float scale_log2;        // softmax scale * log2(e)
 };

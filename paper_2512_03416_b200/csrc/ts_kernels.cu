@@ -524,6 +524,7 @@ extern "C" int ts_decode_attention_static(int32_t device, int32_t n_q_heads, int
   d.table = (int32_t*)block_tables;       // only read
   d.status = &sc->status;
   d.pf_queue = nullptr;
+  d.append_in_decode = 0;
   d.part_acc = sc->part_acc;
   d.part_ml = sc->part_ml;
   d.row_slot = sc->row_slot;
