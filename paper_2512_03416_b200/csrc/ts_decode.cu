@@ -1,5 +1,6 @@
 // Stand-alone split-KV flash-decode kernel for the 1-token rows (sm_100a): one persistent CTA
 // per SM running dec::decode_units (ts_decode_body.h) over all decode units of the step.
+// On a decode-only step (StepDevice::append_in_decode) the units also append the rows' new K/V.
 #include "ts_decode_body.h"
 
 namespace ts {
