@@ -178,11 +178,11 @@ class OracleLeg:
         self.tm = tm
         self.cores = oracle.default_threads()
 
-    def run(self, sel) -> float:
+    def run(self, sel, threads=None) -> float:
         b, s = self.batch, self.batch.shape
         t0 = time.perf_counter()
         self.oracle.attention(self.pool, s.Hq, s.Hkv, s.D, s.P, 1.0 / math.sqrt(s.D), self.tm, b.ctx_len,
-                              b.q_len, b.q, sel=sel, threads=self.cores)
+                              b.q_len, b.q, sel=sel, threads=threads or self.cores)
         return time.perf_counter() - t0
 
     def stride_for(self, seconds: float) -> int:
@@ -220,9 +220,15 @@ def cpu_baseline_leg(batch, target_s: float = 10.0):
     while t < target_s * 0.6 and reps < 64:          # repeat small workloads up to a few seconds of CPU work
         t += leg.run(sel)
         reps += 1
+    # the same oracle on one thread, on a sample thinned by the core count (a few seconds)
+    stride1 = min(max(1, stride * leg.cores * 2), max(1, batch.n_tokens))
+    sel1 = oracle_sample(batch, stride1)
+    t1 = leg.run(sel1, threads=1)
     return {"value": reps * len(sel) / t, "unit": UNIT, "cores": leg.cores, "kind": "oracle",
             "sample": f"every {stride}th decode row and every {stride}th prefill token of {batch.name} "
-                      f"({len(sel)} of {batch.n_tokens} tokens), repeated {reps}x, {t:.1f} s"}
+                      f"({len(sel)} of {batch.n_tokens} tokens), repeated {reps}x, {t:.1f} s",
+            "single_thread": {"value": len(sel1) / t1, "unit": UNIT, "cores": 1,
+                              "sample": f"every {stride1}th decode row and prefill token ({len(sel1)} tokens), {t1:.1f} s"}}
 
 
 def run_reference(args):
@@ -255,7 +261,7 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------- our arm
-def rooflines(peaks, peak_kind, flops, byts, step_ms, prof, parts, traffic=None):
+def rooflines(peaks, peak_kind, flops, byts, step_ms, prof, parts, traffic=None, launches_per_step=None):
     """Roofline of the dominant kernel (times from the library's own CUDA events) and of the step.
 
     `parts` holds algorithmic work per recorded step, averaged over all recorded steps:
@@ -269,6 +275,12 @@ def rooflines(peaks, peak_kind, flops, byts, step_ms, prof, parts, traffic=None)
     dec_ms, pf_ms, mixed_ms = prof["decode_ms"] / steps, prof["prefill_ms"] / steps, prof.get("mixed_ms", 0.0) / steps
     t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
     t_tc = flops / (peaks["bf16_tflops"] * 1e12)
+    # A step that is a single launch: the kernel's average duration is the step time of the timed
+    # region itself (back-to-back launches); the event-per-kernel pass is only needed to split
+    # steps of several launches, and its extra events make each kernel a little slower.
+    source = "events around each kernel, separate pass"
+    if launches_per_step == 1 and mixed_ms > 0:
+        mixed_ms, source = step_ms, "timed region (the launch is the whole step)"
 
     def hbm(kernel, nbytes, ms, tr=None):
         ach = nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
@@ -289,13 +301,14 @@ def rooflines(peaks, peak_kind, flops, byts, step_ms, prof, parts, traffic=None)
         roof = hbm("decode_kernel", parts["dec_bytes"], dec_ms, traffic)
     else:
         roof = tensor("mixed_kernel (prefill tiles only)", parts["pf_flops"], pf_ms)
-    roof.update({"peak_source": f"of {peak_kind}", "decode_ms": dec_ms, "prefill_ms": pf_ms, "mixed_ms": mixed_ms,
+    roof.update({"peak_source": f"of {peak_kind}", "kernel_ms_source": source, "decode_ms": dec_ms, "prefill_ms": pf_ms, "mixed_ms": mixed_ms,
                  "mixed_steps": prof.get("mixed_steps", 0), "recorded_steps": prof["steps"],
                  "append_ms": prof["append_ms"] / steps, "combine_ms": prof["combine_ms"] / steps,
                  "decode_GBps": parts["dec_bytes"] / (dec_ms * 1e-3) / 1e9 if dec_ms > 1e-3 else None,
                  "prefill_TFLOPs": parts["pf_flops"] / (pf_ms * 1e-3) / 1e12 if pf_ms > 1e-3 else None,
                  "mixed_GBps": parts["mixed_bytes"] / (mixed_ms * 1e-3) / 1e9 if mixed_ms > 1e-3 else None,
                  "mixed_TFLOPs": parts["mixed_flops"] / (mixed_ms * 1e-3) / 1e12 if mixed_ms > 1e-3 else None})
+    roof["frac_nominal"] = roof["achieved"] / (8000.0 if roof["bound"] == "hbm" else 2250.0)
     t_roof = max(t_hbm, t_tc)
     step_roof = {"t_roof_us": t_roof * 1e6, "t_hbm_us": t_hbm * 1e6, "t_tensor_us": t_tc * 1e6,
                  "frac": t_roof / (step_ms * 1e-3), "flops": flops, "bytes": byts,
@@ -303,11 +316,20 @@ def rooflines(peaks, peak_kind, flops, byts, step_ms, prof, parts, traffic=None)
     return roof, step_roof
 
 
-def run_static(args, world, rank, local, barrier):
+MIN_TIMED_S = 0.4          # the timed region lasts at least this long, whatever --steps says
+MAX_BLOCKS = 4000
+
+
+def run_static(args, world, rank, local, barrier, workload=None, light=False):
+    """Times blocks of exactly K steps (CUDA events around each block, barrier on both sides of
+    the region), repeated until the region has lasted MIN_TIMED_S, and reports the median block:
+    a handful of 0.16 ms steps is too short a region for the clocks to be sampled or trusted.
+    `light`: no end-to-end leg (the extra workloads of the default line)."""
     import torch
     from paper_2512_03416_b200.harness import LoadedBatch
 
-    batch = make_static_batch(args.workload, rank)
+    workload = workload or args.workload
+    batch = make_static_batch(workload, rank)
     lb = LoadedBatch(batch, device=local, nan_fill=False)
     s = batch.shape
     K, W = args.steps, max(args.warmup, 3)
@@ -317,23 +339,35 @@ def run_static(args, world, rank, local, barrier):
     v0 = lb.dec.velocity()
     sampler = ClockSampler(local)
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    events = [torch.cuda.Event(enable_timing=True)]
     barrier()
-    e0.record()
-    for _ in range(K):
-        lb.step_repeatable()
-    e1.record()
+    t_host = time.perf_counter()
+    events[0].record()
+    n_blocks = 0
+    while True:
+        for _ in range(K):
+            lb.step_repeatable()
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record()
+        events.append(ev)
+        n_blocks += 1
+        if n_blocks % 8 == 0 or n_blocks < 8:
+            ev.synchronize()                          # bounds the queue and gives the region's length so far
+            if time.perf_counter() - t_host >= MIN_TIMED_S or n_blocks >= MAX_BLOCKS:
+                break
     barrier()
     clocks = sampler.stop()
-    ms_step = reduce_max(e0.elapsed_time(e1), world, "cuda") / K
-    launches = int(lb.dec.velocity()["kernel_launches"] - v0["kernel_launches"])
+    block_ms = [events[i].elapsed_time(events[i + 1]) for i in range(n_blocks)]
+    ms_step = reduce_max(float(np.median(block_ms)), world, "cuda") / K
+    region_s = events[0].elapsed_time(events[-1]) * 1e-3
+    launches = int(lb.dec.velocity()["kernel_launches"] - v0["kernel_launches"]) // n_blocks
     tokens = batch.n_tokens
     status = lb.dec.device_status()                   # a bounded wait that ran out would make the timing meaningless
     if status != 0:
         raise SystemExit(f"the device reported status {status} during the timed steps")
 
     lb.dec.profile_enable(True)                       # separate pass: the extra events cost a little
-    for _ in range(min(K, 300)):
+    for _ in range(300):
         lb.step_repeatable()
     prof = lb.dec.profile_read()
     lb.dec.profile_enable(False)
@@ -348,46 +382,56 @@ def run_static(args, world, rank, local, barrier):
              "mixed_bytes": byts if mixed else 0.0,     # the mixed launch also appends the new K/V
              "mixed_flops": flops if mixed else 0.0}
 
-    # end to end: host buffers in, host buffer out, through ts_mixed_step_host
-    Ke = min(K, 300)
-    hq = torch.from_numpy(batch.q.view(np.int16)).pin_memory()
-    hk = torch.from_numpy(batch.k_new.view(np.int16)).pin_memory()
-    hv = torch.from_numpy(batch.v_new.view(np.int16)).pin_memory()
-    ho = torch.empty_like(hq).pin_memory()
-    ql, cl = batch.q_len.tolist(), batch.ctx_len.tolist()
-    for _ in range(3):
-        lb.dec.mixed_step_host(lb.slots, ql, cl, hq, hk, hv, ho, keep_len=True)
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(Ke):         # enqueue only: the next step's upload overlaps this step's kernels and download
-        lb.dec.mixed_step_host(lb.slots, ql, cl, hq, hk, hv, ho, keep_len=True, wait=False)
-    lb.dec.host_fence()
-    torch.cuda.synchronize()
-    e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
-    if lb.dec.device_status() != 0:
-        raise SystemExit("the device reported a failure during the end-to-end loop")
-    e2e = {"value": aggregate_value(tokens, world, e2e_s / Ke), "unit": UNIT,
-           "h2d_bytes_per_step": int(hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2),
-           "d2h_bytes_per_step": int(ho.numel() * 2), "steps": Ke, "ms_per_step": e2e_s / Ke * 1e3}
     kv_tokens = int((batch.ctx_len + batch.q_len).sum())
     cfg = {"decode_rows": batch.decode_tokens, "prefill_tokens": batch.prefill_tokens, "kv_tokens": kv_tokens,
-           "l2": "inputs larger than L2 (KV working set %.2f GB)" % (kv_tokens * s.kv_bytes_per_token / 1e9)}
+           "l2": "inputs larger than L2 (KV working set %.2f GB)" % (kv_tokens * s.kv_bytes_per_token / 1e9),
+           "timing": f"median of {n_blocks} blocks of {K} steps, CUDA events around each block, "
+                     f"timed region {region_s:.2f} s"}
+    e2e = None
+    if not light:
+        # end to end: host buffers in, host buffer out, through ts_mixed_step_host; one pipelined
+        # region of at least K steps and at least MIN_TIMED_S
+        hq = torch.from_numpy(batch.q.view(np.int16)).pin_memory()
+        hk = torch.from_numpy(batch.k_new.view(np.int16)).pin_memory()
+        hv = torch.from_numpy(batch.v_new.view(np.int16)).pin_memory()
+        ho = torch.empty_like(hq).pin_memory()
+        ql, cl = batch.q_len.tolist(), batch.ctx_len.tolist()
+        t0 = time.perf_counter()
+        for _ in range(3):
+            lb.dec.mixed_step_host(lb.slots, ql, cl, hq, hk, hv, ho, keep_len=True)
+        est = (time.perf_counter() - t0) / 3
+        Ke = int(min(max(K, math.ceil(MIN_TIMED_S / max(est, 1e-5))), 5000))
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(Ke):         # enqueue only: the next step's upload overlaps this step's kernels and download
+            lb.dec.mixed_step_host(lb.slots, ql, cl, hq, hk, hv, ho, keep_len=True, wait=False)
+        lb.dec.host_fence()
+        torch.cuda.synchronize()
+        e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
+        if lb.dec.device_status() != 0:
+            raise SystemExit("the device reported a failure during the end-to-end loop")
+        e2e = {"value": aggregate_value(tokens, world, e2e_s / Ke), "unit": UNIT,
+               "h2d_bytes_per_step": int(hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2),
+               "d2h_bytes_per_step": int(ho.numel() * 2), "steps": Ke, "ms_per_step": e2e_s / Ke * 1e3}
+    lb.dec.close()
     return dict(batch=batch, ms_step=ms_step, tokens=tokens, prefill_tokens=batch.prefill_tokens,
                 decode_tokens=batch.decode_tokens, launches=launches, clocks=clocks, prof=prof, flops=flops,
-                byts=byts, parts=parts, e2e=e2e, cfg=cfg, steps=K, warmup=W, extra={})
+                byts=byts, parts=parts, e2e=e2e, cfg=cfg, steps=K, warmup=W,
+                extra={"timed_blocks": n_blocks, "timed_region_s": region_s})
 
 
-def run_replay(args, world, rank, local, barrier):
+def run_replay(args, world, rank, local, barrier, workload=None, light=False, n_steps=None):
     """config5: the 200-step bursty replay. Every step is issued once, in order (the state evolves);
-    warm-up is a full untimed replay on a fresh instance."""
+    warm-up is a full untimed replay on a fresh instance. `light`: no end-to-end leg."""
     import torch
     from paper_2512_03416_b200.replay import ReplayRunner, ttft_report
 
-    K = min(args.steps, 200)
+    workload = workload or args.workload
+    K = n_steps or min(args.steps, 200)
     seed = rank_seed(5, rank)
 
     def fresh(keep_host=False):
-        return ReplayRunner(wl.TraceReplay(seed=seed, n_steps=K, **REPLAY_TRACE[args.workload]), seed=seed + 45,
+        return ReplayRunner(wl.TraceReplay(seed=seed, n_steps=K, **REPLAY_TRACE[workload]), seed=seed + 45,
                             device=local, keep_host=keep_host)
 
     warm = fresh()
@@ -443,35 +487,37 @@ def run_replay(args, world, rank, local, barrier):
     parts = {"dec_bytes": dec_bytes / n_rec, "pf_flops": pf_flops / n_rec, "mixed_bytes": mixed_bytes / n_rec,
              "mixed_flops": mixed_flops / n_rec}
 
-    # end to end: every step's inputs start in pinned host memory and its output returns there
-    e2e_run = fresh(keep_host=True)
-    pinned = []
-    for ps in e2e_run.steps:
-        if ps.host is None:
-            pinned.append(None)
-            continue
-        hq, hk, hv = (torch.from_numpy(a.view(np.int16)).pin_memory() for a in ps.host)
-        pinned.append((hq, hk, hv, torch.empty_like(hq).pin_memory()))
-    e2e_run.start()
-    barrier()
-    t0 = time.perf_counter()
-    h2d = d2h = 0
-    for ps, pin in zip(e2e_run.steps, pinned):
-        e2e_run.begin_step(ps)
-        if pin is not None:
-            hq, hk, hv, ho = pin
-            e2e_run.dec.mixed_step_host(ps.slots.tolist(), ps.q_len, ps.ctx_len, hq, hk, hv, ho, wait=False)
-            h2d += (hq.numel() + hk.numel() + hv.numel()) * 2
-            d2h += ho.numel() * 2
-        e2e_run.end_step(ps)
-    e2e_run.dec.host_fence()
-    torch.cuda.synchronize()
-    e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
-    if e2e_run.dec.device_status() != 0:
-        raise SystemExit("the device reported a failure during the end-to-end replay")
-    e2e_run.dec.close()
-    e2e = {"value": aggregate_value(tokens, world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": int(h2d / K),
-           "d2h_bytes_per_step": int(d2h / K), "steps": K, "ms_per_step": e2e_s / K * 1e3}
+    e2e = None
+    if not light:
+        # end to end: every step's inputs start in pinned host memory and its output returns there
+        e2e_run = fresh(keep_host=True)
+        pinned = []
+        for ps in e2e_run.steps:
+            if ps.host is None:
+                pinned.append(None)
+                continue
+            hq, hk, hv = (torch.from_numpy(a.view(np.int16)).pin_memory() for a in ps.host)
+            pinned.append((hq, hk, hv, torch.empty_like(hq).pin_memory()))
+        e2e_run.start()
+        barrier()
+        t0 = time.perf_counter()
+        h2d = d2h = 0
+        for ps, pin in zip(e2e_run.steps, pinned):
+            e2e_run.begin_step(ps)
+            if pin is not None:
+                hq, hk, hv, ho = pin
+                e2e_run.dec.mixed_step_host(ps.slots.tolist(), ps.q_len, ps.ctx_len, hq, hk, hv, ho, wait=False)
+                h2d += (hq.numel() + hk.numel() + hv.numel()) * 2
+                d2h += ho.numel() * 2
+            e2e_run.end_step(ps)
+        e2e_run.dec.host_fence()
+        torch.cuda.synchronize()
+        e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
+        if e2e_run.dec.device_status() != 0:
+            raise SystemExit("the device reported a failure during the end-to-end replay")
+        e2e_run.dec.close()
+        e2e = {"value": aggregate_value(tokens, world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": int(h2d / K),
+               "d2h_bytes_per_step": int(d2h / K), "steps": K, "ms_per_step": e2e_s / K * 1e3}
     order = np.argsort(step_ms)
     heavy = [i for i in range(K) if run.steps[i].prefill_tokens >= 4096]
     extra = {"step_ms": {"median": float(np.median(step_ms)), "p90": float(np.percentile(step_ms, 90)),
@@ -509,10 +555,35 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    r = (run_replay if args.workload in REPLAY_TRACE else run_static)(args, world, rank, local, barrier)
     peaks, peak_kind = load_peaks()
-    roofline, step_roofline = rooflines(peaks, peak_kind, r["flops"], r["byts"], r["ms_step"], r["prof"], r["parts"],
-                                        KERNEL_TRAFFIC_BYTES.get(args.workload))
+
+    def measure(workload, light, n_steps=None):
+        if workload in REPLAY_TRACE:
+            r = run_replay(args, world, rank, local, barrier, workload, light, n_steps)
+        else:
+            r = run_static(args, world, rank, local, barrier, workload, light)
+        lps = r["launches"] / max(1, r["steps"]) if r["batch"] is not None else None
+        roof, step_roof = rooflines(peaks, peak_kind, r["flops"], r["byts"], r["ms_step"], r["prof"], r["parts"],
+                                    KERNEL_TRAFFIC_BYTES.get(workload), launches_per_step=lps)
+        return r, roof, step_roof
+
+    r, roofline, step_roofline = measure(args.workload, light=False)
+    # The default line also carries short passes of the other target workloads (no end-to-end and
+    # no oracle leg for them): the decode-only batch, the chunked continuation and the 200-step
+    # 70B-shaped replay.
+    others = {}
+    if args.workload == "config3" and not args.headline_only and world == 1:
+        for w in ("config2", "config4", "config5"):
+            ro, roofo, stepo = measure(w, light=True, n_steps=200 if w in REPLAY_TRACE else None)
+            others[w] = {"description": WORKLOADS[w][1], "ms_per_step": ro["ms_step"], "steps": ro["steps"],
+                         "tokens_per_s": aggregate_value(ro["tokens"], world, ro["ms_step"] * 1e-3),
+                         "step_roofline": {k: stepo[k] for k in ("frac", "frac_nominal", "t_roof_us", "t_hbm_us", "t_tensor_us")},
+                         "roofline": {k: roofo[k] for k in ("kernel", "bound", "achieved", "peak", "unit", "frac",
+                                                             "frac_nominal", "kernel_ms", "kernel_ms_source", "peak_source")},
+                         "clocks": ro["clocks"], "gpu_launches": ro["launches"]}
+            for k in ("heavy_steps", "sum_t_roof_over_sum_t", "step_ms", "timed_blocks", "timed_region_s"):
+                if k in ro["extra"]:
+                    others[w][k] = ro["extra"][k]
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = cpu_baseline_leg(r["batch"] if r["batch"] is not None else make_static_batch(args.workload, 0))
@@ -531,6 +602,8 @@ def run_ours(args):
                 "prefill_tokens_per_s": aggregate_value(r["prefill_tokens"], world, r["ms_step"] * 1e-3),
                 "decode_tokens_per_s": aggregate_value(r["decode_tokens"], world, r["ms_step"] * 1e-3)}
         line.update(r["extra"])
+        if others:
+            line["workloads"] = others
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -544,6 +617,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config3", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="default workload only: skip the short passes of config2, config4 and config5")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -97,7 +97,21 @@ typedef struct {
                                  256-byte aligned; holds the device block table, the step
                                  metadata, split partials and the host-buffer staging area     */
   size_t workspace_bytes;
+  int64_t wait_limit_cycles;  /* limit of every bounded wait inside the kernels, in GPU clock
+                                 cycles; 0 = the library's default (about one second)          */
+  int32_t debug_flags;        /* 0, or TS_DEBUG_* bits (testing the failure path, see below)   */
 } ts_config;
+
+/*
+ * Debug flags (the paper has no counterpart). TS_DEBUG_LOSE_APPEND_ARRIVAL makes the launch-wide
+ * barrier after the KV append of a step with prefill rows wait for one thread block more than the
+ * launch has, so that this wait runs out: every block then raises TS_DEV_TIMEOUT after
+ * wait_limit_cycles and carries on (all blocks did arrive, so the step's output is still valid).
+ * It exists so that the time-out path can be exercised without a fault: ts_create refuses it
+ * (TS_ERR_INVALID) unless 0 < wait_limit_cycles <= 50,000,000 (about 25 ms), so it can never spin
+ * for the default second.
+ */
+enum { TS_DEBUG_LOSE_APPEND_ARRIVAL = 1 };
 
 /* Sizes the caller must allocate. Only the shape fields of cfg are read. 0 on a bad shape. */
 size_t ts_pool_bytes(const ts_config* cfg);
@@ -374,7 +388,7 @@ int ts_last_device_status(ts_ctx* ctx, void* cuda_stream, int32_t* status_out);
  * handed tensors and is not allowed to own memory; or a latency-critical loop that cannot
  * afford the device-wide synchronisation an allocation may imply. Such a caller cannot supply
  * the workspace ts_create asks for. Here the split partials and the work list live in a
- * fixed array inside the library (about 8.6 MiB, present on every GPU that loads the
+ * fixed array inside the library (about 8.4 MiB, present on every GPU that loads the
  * library, until the process ends). The call makes no cudaMalloc/cudaFree and uses no
  * allocating routine.
  *
@@ -382,7 +396,10 @@ int ts_last_device_status(ts_ctx* ctx, void* cuda_stream, int32_t* status_out);
  *   kv_pool       the pool in the layout documented above; the K/V of every attended token,
  *                 the newest one included, must already be in it (this call appends nothing)
  *   block_tables  int32 [n_rows][table_width]: page ids of row r in its first
- *                 ceil(kv_len[r]/16) entries
+ *                 ceil(kv_len[r]/16) entries. A page id outside [0, n_pages) is not followed:
+ *                 its 16 keys count as absent (zero-filled K/V), the row's output is then wrong
+ *                 but finite, and NO error is reported -- this entry point has no status word
+ *                 the host can read, so the caller must pass valid tables
  *   kv_len        int32 [n_rows]: tokens row r attends to, 1 <= kv_len[r] <= 16*table_width
  *                 (a row outside this range is not processed and its output is NaN)
  *   q, out        bf16 [n_rows, n_q_heads, head_dim], 16-byte aligned

@@ -26,6 +26,7 @@ TS_STEP_HOST_ASYNC = 2
 TS_DEV_BAD_PAGE = 1
 TS_DEV_TIMEOUT = 2
 TS_DEV_BAD_INDEX = 4
+TS_DEBUG_LOSE_APPEND_ARRIVAL = 1
 
 _i32p = ctypes.POINTER(ctypes.c_int32)
 
@@ -39,7 +40,8 @@ class ts_config(ctypes.Structure):
                 ("mixed_prefill_ctas", ctypes.c_int32), ("softmax_scale", ctypes.c_float), ("device", ctypes.c_int32),
                 ("alloc_shuffle_seed", ctypes.c_uint64),
                 ("kv_pool", ctypes.c_void_p), ("kv_pool_bytes", ctypes.c_size_t),
-                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+                ("wait_limit_cycles", ctypes.c_int64), ("debug_flags", ctypes.c_int32)]
 
 
 class ts_step(ctypes.Structure):

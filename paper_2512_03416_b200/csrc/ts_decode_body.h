@@ -209,7 +209,7 @@ __device__ __forceinline__ void decode_units(const StepDevice& s, const CUtensor
       const int stage = n_consumed % STAGES;
       const uint32_t parity = (n_consumed / STAGES) & 1;
       const uint32_t sp = ring + stage * STAGE_BYTES;
-      if (!mbar_wait(my_bars + stage * 8, parity, dead ? 1000 : kWaitCycles)) {
+      if (!mbar_wait(my_bars + stage * 8, parity, dead ? 1000 : s.wait_cycles)) {
         if (!dead && lane == 0) atomicOr(s.status, TS_DEV_TIMEOUT);
         dead = true;
       }

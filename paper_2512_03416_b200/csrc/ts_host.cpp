@@ -46,6 +46,7 @@ bool shape_ok(const ts_config* c) {
   if (c->n_q_heads / c->n_kv_heads > ts::kMaxGroup) return false;
   if (c->n_pages <= 0 || c->max_requests <= 0 || c->max_pages_per_req <= 0) return false;
   if (c->chunk_size < 0 || c->reserved_pages < 0 || c->decode_split_tokens < 0) return false;
+  if (c->wait_limit_cycles < 0) return false;
   return true;
 }
 
@@ -156,6 +157,7 @@ struct ts_ctx {
   std::vector<CombineItem> combines;
   std::vector<int32_t> tok0;
   std::vector<TableDelta> deltas;
+  std::vector<std::pair<int32_t, int32_t>> sync_marks;   // (slot, table entries the device will hold)
   // optional per-kernel timing: 5 events per recorded step
   bool profiling = false;
   std::vector<cudaEvent_t> prof_events;
@@ -373,12 +375,15 @@ void plan(ts_ctx* c, const ts_step* st) {
 int sync_tables(ts_ctx* c, const ts_step* st, cudaStream_t stream, int* n_slot_deltas) {
   *n_slot_deltas = 0;
   c->deltas.clear();
+  c->sync_marks.clear();
   for (int r = 0; r < st->n_rows; ++r) {
     Slot& s = c->slots[st->slot[r]];
     const int32_t* row = table_row(c, st->slot[r]);
     for (int i = s.synced_pages; i < s.n_pages; ++i)
       c->deltas.push_back(TableDelta{st->slot[r], i, row[i]});
-    s.synced_pages = s.n_pages;
+    // synced_pages only advances once the entries are on their way (commit_table_sync): a step
+    // that fails before that leaves the record as it was, and the next step sends them again
+    if (s.n_pages > s.synced_pages) c->sync_marks.push_back({st->slot[r], s.n_pages});
   }
   if (c->deltas.size() <= (size_t)kSlotDeltas) {
     // the usual case (a few rows crossed a page boundary): the entries travel with the step's
@@ -403,6 +408,12 @@ int sync_tables(ts_ctx* c, const ts_step* st, cudaStream_t stream, int* n_slot_d
     at += n;
   }
   return TS_OK;
+}
+
+// The table entries gathered by sync_tables have been enqueued (copy and table_update launch).
+void commit_table_sync(ts_ctx* c) {
+  for (const auto& m : c->sync_marks) c->slots[m.first].synced_pages = m.second;
+  c->sync_marks.clear();
 }
 
 // Sends the step's metadata to the next device slot. The copy goes over the context's copy stream:
@@ -493,6 +504,8 @@ void fill_device(ts_ctx* c, const ts_step* st, int64_t n_tokens, ts::StepDevice*
   d->max_requests = c->cfg.max_requests;
   d->scale_log2 = c->scale * 1.4426950408889634f;
   d->append_in_decode = 0;
+  d->wait_cycles = c->cfg.wait_limit_cycles > 0 ? (long long)c->cfg.wait_limit_cycles : ts::kWaitCycles;
+  d->append_arrivals = 0;      // set by the mixed launch
 }
 
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
@@ -570,6 +583,7 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
   const int n_combines = attention ? (int)c->combines.size() : 0;
   rc = upload_meta(c, st, n_items, n_combines, n_slot_deltas, stream);
   if (rc != TS_OK) return rc;
+  commit_table_sync(c);
   ts::StepDevice d;
   fill_device(c, st, n_tokens, &d);
   d.n_items = n_items;
@@ -630,6 +644,7 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
           decode_launched = true;
         }
         if (pe) c->prof_mixed.back() = decode_launched;
+        d.append_arrivals = n_ctas + ((c->cfg.debug_flags & TS_DEBUG_LOSE_APPEND_ARRIVAL) ? 1 : 0);
         TS_CUDA(c, ts::launch_mixed(d, q_map, c->kv_map, n_ctas, p, stream));
       } else {
         ts::StepDevice dp = d;
@@ -683,6 +698,10 @@ int ts_create(const ts_config* cfg, ts_ctx** out) {
   if (!cfg) return TS_ERR_INVALID;
   if (!shape_ok(cfg)) return TS_ERR_UNSUPPORTED;
   if (cfg->reserved_pages > cfg->n_pages) return TS_ERR_INVALID;
+  if (cfg->debug_flags & ~TS_DEBUG_LOSE_APPEND_ARRIVAL) return TS_ERR_INVALID;
+  if ((cfg->debug_flags & TS_DEBUG_LOSE_APPEND_ARRIVAL) &&
+      (cfg->wait_limit_cycles <= 0 || cfg->wait_limit_cycles > 50000000))
+    return TS_ERR_INVALID;    // a wait that is meant to run out must be short
   Layout L;
   compute_layout(cfg, &L);
   if (cfg->kv_pool && cfg->kv_pool_bytes < ts_pool_bytes(cfg)) return TS_ERR_WORKSPACE;
@@ -873,6 +892,13 @@ int ts_mixed_step_host(ts_ctx* c, const ts_step* st, void* cuda_stream) {
   }
   if (!st->q || !st->k_new || !st->v_new || !st->out) return TS_ERR_INVALID;
   if (!c->cfg.workspace) return cuda_fail(c, cudaErrorInvalidDevicePointer);
+  {
+    // the step's own checks first: a step that would be refused must not start copying
+    int64_t nt = 0, np = 0;
+    int nd = 0;
+    const int vrc = validate(c, st, true, true, &nt, &nd, &np);
+    if (vrc != TS_OK) return vrc;
+  }
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   TS_CUDA(c, cudaSetDevice(c->cfg.device));
   if (!c->up_stream) {

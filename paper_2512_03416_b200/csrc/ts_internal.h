@@ -15,6 +15,7 @@ constexpr int kPageSize = 16;
 constexpr int kKeysPerTile = 64;     // keys staged per pipeline stage of the attention kernel
 constexpr int kPackedRowsPerTile = 64;  // (token, head) rows of a prefill tile, head_dim 64 path
 constexpr int kPackedRowsTc = 128;      // (token, head) rows of a prefill tile, tcgen05 path (head_dim 128)
+constexpr long long kWaitCycles = 2000000000LL;  // default limit of a bounded wait: about one second at boost clock
 constexpr int kMaxGroup = 16;        // query heads per KV head a decode work item can hold
 
 // One unit of attention work; the KV head comes from the grid.
@@ -74,6 +75,9 @@ struct StepDevice {
   int32_t append_in_decode; // != 0: the decode units append their rows' new K/V themselves
   int32_t Hq, Hkv, D, n_pages, max_pages_per_req, max_requests;
   float scale_log2;        // softmax scale * log2(e)
+  long long wait_cycles;   // limit of every bounded wait of the step's kernels, in clock cycles
+  int32_t append_arrivals; // CTAs the mixed kernel's append barrier waits for: its grid size, or one
+                           // more when ts_config.debug_flags asks for a wait that runs out
 };
 
 // Launchers. Each enqueues on `stream` and returns the launch's cudaError_t.

@@ -1,10 +1,11 @@
 // CUDA kernels (sm_100a) of the mixed paged-attention step:
 //   table_update  - applies block-table deltas to the device copy of the tables
 //   kv_append     - copies the step's new K/V into their pages (16-byte vector copies)
-//   attention     - one launch for both row kinds: split-KV flash-decode work items for the
-//                   1-token rows and causal tiles for the prefill-chunk rows, K/V pages staged
-//                   in shared memory through a 3-stage cp.async ring, bf16 tensor-core MMAs with
-//                   fp32 online softmax (warp-shuffle reductions)
+//   attention     - prefill tiles of head_dim 64 steps, and the kernel behind
+//                   ts_decode_attention_static (decode work items): K/V pages staged in shared
+//                   memory through a 3-stage cp.async ring, mma.sync bf16 MMAs with fp32 online
+//                   softmax (warp-shuffle reductions). head_dim 128 steps run ts_mixed.cu and
+//                   ts_decode.cu instead.
 //   combine       - log-sum-exp merge of the decode splits
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -430,7 +431,7 @@ struct StaticScratch {
   int32_t status;
 };
 
-// Lives in every context that loads the library, until the process exits (about 8.6 MiB).
+// Lives in every context that loads the library, until the process exits (about 8.4 MiB).
 static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
 
 // One thread per (row, split): writes the row arrays, the work items and the combine list.

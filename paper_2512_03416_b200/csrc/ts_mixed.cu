@@ -323,7 +323,7 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
     }
   };
   auto wait = [&](int i, uint32_t parity) {
-    if (!mbar_wait(bar(i), parity, misc[1] ? 2000 : kWaitCycles)) give_up();
+    if (!mbar_wait(bar(i), parity, misc[1] ? 2000 : s.wait_cycles)) give_up();
   };
   // k-th work unit of this CTA (w = -1 after the last one), published by the K loaders' first thread
   volatile int4* ring = reinterpret_cast<volatile int4*>(smem + kOffRing);
@@ -331,7 +331,7 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
     if ((int)misc[2] <= k) {
       const long long t0 = clock64();
       while ((int)misc[2] <= k) {
-        if (clock64() - t0 > (misc[1] ? 2000 : kWaitCycles)) {
+        if (clock64() - t0 > (misc[1] ? 2000 : s.wait_cycles)) {
           give_up();
           return false;
         }
@@ -361,6 +361,18 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
       mbar_init_fence();
     }
     if (warp == kWarpMma) tmem_alloc(base + kOffMisc, 512);
+    // When G does not divide 128 a query tile holds tile_tokens * G < 128 packed rows and the Q
+    // copies never write the rest: clear those rows once, so that the MMA reads zeros there and
+    // not whatever the shared memory held before.
+    const int used_rows = tile_tokens * G;
+    if (used_rows < 128) {
+      const int n16 = (128 - used_rows) * 8;                 // 16-byte chunks per 64-column half tile
+      for (int i = tid; i < 4 * n16; i += kPfThreads) {
+        const int half = i / n16, c = i % n16;
+        *reinterpret_cast<uint4*>(smem + kOffQ + half * kHalfBytes + used_rows * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+      }
+      fence_proxy_async();
+    }
     tc_fence_before();
     cta_sync();
     tc_fence_after();
@@ -387,8 +399,8 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
       atomicAdd(s.pf_queue + 2, 1);
       const volatile int32_t* arrived = s.pf_queue + 2;
       const long long t0 = clock64();
-      while (*arrived < (int)gridDim.x) {
-        if (clock64() - t0 > kWaitCycles) {
+      while (*arrived < s.append_arrivals) {
+        if (clock64() - t0 > s.wait_cycles) {
           atomicOr(s.status, TS_DEV_TIMEOUT);
           break;
         }
@@ -534,7 +546,7 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
         const volatile int32_t* done = s.pf_queue + 1;
         const long long t0 = clock64();
         while (*done < n_decode_ctas) {
-          if (clock64() - t0 > (misc[1] ? 2000 : kWaitCycles)) {
+          if (clock64() - t0 > (misc[1] ? 2000 : s.wait_cycles)) {
             give_up();
             break;
           }
@@ -701,7 +713,7 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
       // the warp keeps its own failure flag in a register: nothing on its path reads shared memory
       bool dead = false;
       auto iwait = [&](int i, uint32_t parity) {
-        if (!mbar_wait(bar(i), parity, dead ? 2000 : kWaitCycles)) {
+        if (!mbar_wait(bar(i), parity, dead ? 2000 : s.wait_cycles)) {
           dead = true;
           give_up();
         }
@@ -790,7 +802,8 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
         if (!get_work(k, u)) break;
         const int ta = u.tok0 + u.q_begin;
         if (k > 0) wait(BAR_Q_EMPTY, (k - 1) & 1);
-        mbar_expect_tx(bar(BAR_Q), (u.cnt_b > 0 ? 2 : 1) * kTileBytes);
+        // a box delivers 64 columns of tile_tokens * G packed rows (all 128 only when G divides 128)
+        mbar_expect_tx(bar(BAR_Q), (u.cnt_b > 0 ? 2 : 1) * 2 * (tile_tokens * G * 128));
         tma_load_4d(base + kOffQ, &q_map, bar(BAR_Q), 0, 0, u.kv_head, ta);
         tma_load_4d(base + kOffQ + kHalfBytes, &q_map, bar(BAR_Q), 64, 0, u.kv_head, ta);
         if (u.cnt_b > 0) {

@@ -1,13 +1,14 @@
 // Device-side helpers for TMA tensor copies and mbarriers (sm_100a, inline PTX).
-// Every wait is bounded: it gives up after kWaitCycles clock cycles and reports failure, so a
+// Every wait is bounded: it gives up after its limit of clock cycles (kWaitCycles unless the
+// context sets its own) and reports failure, so a
 // lost copy or a protocol mistake ends the kernel with an error flag instead of a hang.
 #pragma once
 #include <cuda.h>
 #include <stdint.h>
 
-namespace ts {
+#include "ts_internal.h"
 
-constexpr long long kWaitCycles = 2000000000LL;  // about one second at boost clock
+namespace ts {
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");

@@ -36,13 +36,14 @@ class Decoder:
                  max_pages_per_req: int, chunk_size: int = 0, reserved_pages: int = 0,
                  decode_split_tokens: int = 0, softmax_scale: float = 0.0, device: int = 0,
                  alloc_shuffle_seed: int = 0, page_size: int = 16, nan_fill: bool = False,
-                 mixed_prefill_ctas: int = 0):
+                 mixed_prefill_ctas: int = 0, wait_limit_cycles: int = 0, debug_flags: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required; there is no CPU implementation")
         self.device = torch.device("cuda", device)
         cfg = B.ts_config(n_q_heads, n_kv_heads, head_dim, page_size, n_pages, max_requests,
                           max_pages_per_req, chunk_size, reserved_pages, decode_split_tokens,
-                          mixed_prefill_ctas, softmax_scale, device, alloc_shuffle_seed, None, 0, None, 0)
+                          mixed_prefill_ctas, softmax_scale, device, alloc_shuffle_seed, None, 0, None, 0,
+                          wait_limit_cycles, debug_flags)
         pool_bytes, ws_bytes = B.ts_pool_bytes(cfg), B.ts_workspace_bytes(cfg)
         if pool_bytes == 0:
             raise TsError(B.TS_ERR_UNSUPPORTED, "ts_pool_bytes")

@@ -25,7 +25,7 @@ class LoadedBatch:
 
     def __init__(self, batch: wl.StepBatch, decode_split_tokens: int = 0, chunk_size=None,
                  max_requests=None, extra_pages: int = 0, device: int = 0, nan_fill: bool = True,
-                 mixed_prefill_ctas: int = 0):
+                 mixed_prefill_ctas: int = 0, wait_limit_cycles: int = 0, debug_flags: int = 0):
         s = batch.shape
         width = max([len(t) for t in batch.tables] + [1]) + extra_pages
         cs = batch.chunk_size if chunk_size is None else chunk_size
@@ -33,7 +33,8 @@ class LoadedBatch:
         self.device = torch.device("cuda", device)
         self.dec = Decoder(s.Hq, s.Hkv, s.D, batch.n_pages, max_requests or max(batch.n_rows, 1), width,
                            chunk_size=cs, decode_split_tokens=decode_split_tokens, device=device,
-                           nan_fill=nan_fill, mixed_prefill_ctas=mixed_prefill_ctas)
+                           nan_fill=nan_fill, mixed_prefill_ctas=mixed_prefill_ctas,
+                           wait_limit_cycles=wait_limit_cycles, debug_flags=debug_flags)
         self.slots = []
         for r in range(batch.n_rows):
             slot = self.dec.request_add(1000 + r, int(batch.ctx_len[r]) + int(batch.q_len[r]))

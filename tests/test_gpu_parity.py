@@ -47,6 +47,18 @@ CASES = [
     (2, 2, 128, [0], [1]),
     (12, 4, 64, [19], [300]),
     (16, 1, 64, [40, 41], [1, 5]),
+    # head_dim 128 with group sizes that do not divide 128 (query tiles of 126, 125, 126, 120 packed rows)
+    (24, 8, 128, [300, 0, 77], [1, 200, 1]),
+    (40, 8, 128, [33, 5], [1, 150]),
+    (48, 8, 128, [129, 600, 18], [140, 1, 1]),
+    (7, 1, 128, [0, 260], [90, 1]),
+    (12, 1, 128, [70, 15, 0], [1, 1, 75]),
+    # sixteen query heads per KV head at head_dim 128: 8-token query tiles, the decode rows in a
+    # launch of their own (two head groups per unit) followed by the split merge
+    (16, 1, 128, [900, 0, 4500, 31], [1, 70, 1, 1]),
+    (32, 2, 128, [257, 5000, 12], [1, 1, 100]),
+    (32, 2, 128, [255, 256, 4700, 0], [1, 1, 1, 1]),
+    (16, 1, 128, [4200, 63], [1, 1]),
 ]
 
 
@@ -89,7 +101,7 @@ def test_config3_burst_8b(profile):
     assert np.array_equal(run.pool(), pool_want)
 
 
-@pytest.mark.parametrize("profile", ["paper", "needle"])
+@pytest.mark.parametrize("profile", ["paper", "peaked", "needle"])
 def test_config4_chunked_8b(profile):
     b = wl.config4(profile=profile)
     want, pool_want = oracle_step(b)
@@ -152,3 +164,33 @@ def test_maximum_sizes_sampled():
     got = run.step()[sel]
     assert_parity(got, want, "peaked", "maximum sizes")
     assert np.array_equal(run.pool(), pool_want)
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_next_step_is_clean():
+    """Failure path without a fault: with TS_DEBUG_LOSE_APPEND_ARRIVAL the barrier after the KV
+    append of a mixed step waits for one thread block more than the launch has, under a limit of
+    2 million clock cycles (about a millisecond; never the library's default second). Every block
+    then gives that wait up, raises TS_DEV_TIMEOUT and carries on. The step must return, the status
+    call must report TS_ERR_DEVICE_TIMEOUT once and then be clean, and a normal context's next
+    step on the same device must match the oracle, pool included."""
+    from paper_2512_03416_b200 import binding as B
+    b = wl.make_batch("tmo", wl.LLAMA8B, [300, 40, 0], [1, 1, 300], seed=41, profile="peaked")
+    want, pool_want = oracle_step(b)
+    run = GpuRun(b, chunk_size=0, wait_limit_cycles=2_000_000, debug_flags=B.TS_DEBUG_LOSE_APPEND_ARRIVAL)
+    run.lb.step(keep_len=True)
+    rc, bits = B.ts_last_device_status(run.dec.ctx, torch.cuda.current_stream().cuda_stream)
+    assert rc == B.TS_ERR_DEVICE_TIMEOUT and bits & B.TS_DEV_TIMEOUT
+    # all blocks had in fact arrived, so even this step's result is complete
+    assert_parity(run.lb.output(), want, "peaked", "step whose append barrier gave up")
+    rc, bits = B.ts_last_device_status(run.dec.ctx, torch.cuda.current_stream().cuda_stream)
+    assert rc == B.TS_OK and bits == 0, "the status word was not cleared"
+    # the launch's counters are back at zero: the same context runs the step again, still flagged
+    run.lb.step(keep_len=True)
+    assert run.dec.device_status() == B.TS_DEV_TIMEOUT
+    run.dec.close()
+    # and a context without the flag is clean
+    ok = GpuRun(b, chunk_size=0)
+    got = ok.step()
+    assert_parity(got, want, "peaked", "step after a timed-out one")
+    assert np.array_equal(ok.pool(), pool_want)
+

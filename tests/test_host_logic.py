@@ -311,3 +311,19 @@ def test_scaler_and_router_match_the_oracle():
     assert B.ts_decoder_demand([1.0], [0.0]) == -1.0
     assert B.ts_regular_decoders(0.0, 1) == 0
     assert B.ts_route_prefill([1.0], [0.0], [], [], 1.0)[0] == B.TS_ERR_INVALID
+
+
+def test_debug_flag_needs_a_short_wait_limit():
+    """The flag that makes a wait run out is refused unless the context's wait limit is short."""
+    for limit in (0, 50_000_001):
+        cfg = B.ts_config(32, 8, 128, 16, 100, 8, 64, 0, 0, 0, 0, 0.0, 0, 0, None, 0, None, 0, limit,
+                          B.TS_DEBUG_LOSE_APPEND_ARRIVAL)
+        rc, _ = B.ts_create(cfg)
+        assert rc == B.TS_ERR_INVALID
+    cfg = B.ts_config(32, 8, 128, 16, 100, 8, 64, 0, 0, 0, 0, 0.0, 0, 0, None, 0, None, 0, 2_000_000,
+                      B.TS_DEBUG_LOSE_APPEND_ARRIVAL)
+    rc, h = B.ts_create(cfg)
+    assert rc == B.TS_OK
+    B.ts_destroy(h)
+    cfg.debug_flags = 2                      # unknown bit
+    assert B.ts_create(cfg)[0] == B.TS_ERR_INVALID

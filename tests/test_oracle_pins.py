@@ -125,6 +125,36 @@ def pin_matches_library_attention_fp64():
             assert err <= tol, f"{shape} row {row}: {err}"
 
 
+def pin_selected_tokens_are_the_named_ones():
+    """The `sel` form returns, in the order of `sel` (shuffled, with a repeat), exactly what the
+    full call returns for those tokens, and each selected token matches a direct fp64 softmax
+    over its own row's gathered keys: the index goes to the right row, position and output slot."""
+    s = wl.Shape(6, 2, 64)
+    ctx, ql = [9, 40, 0, 21], [1, 1, 35, 18]
+    b = wl.make_batch("t", s, ctx, ql, seed=77, profile="peaked")
+    full, _ = oracle_step(b)
+    rng = np.random.default_rng(3)
+    sel = rng.permutation(b.n_tokens)[:23].astype(np.int32)
+    sel = np.concatenate([sel, sel[:1], [0, b.n_tokens - 1]]).astype(np.int32)
+    got, _ = oracle_step(b, sel=sel)
+    assert got.shape == (len(sel), s.Hq, s.D)
+    assert np.array_equal(got, full[sel])
+    starts = np.concatenate([[0], np.cumsum(ql)])
+    for o, tok in enumerate(sel.tolist()):
+        r = int(np.searchsorted(starts, tok, side="right") - 1)
+        i = tok - int(starts[r])
+        k, v = gathered_kv(b, r)                                          # [n, Hkv, D] fp64
+        n = ctx[r] + i + 1
+        for h in range(s.Hq):
+            g = h // s.G
+            q = f32(b.q[tok, h]).astype(np.float64)
+            sc = (k[:n, g] @ q) / math.sqrt(s.D)
+            w = np.exp(sc - sc.max())
+            ref = (w[:, None] * v[:n, g]).sum(0) / w.sum()
+            assert np.abs(got[o, h] - ref).max() <= 1e-5 * max(1.0, np.abs(ref).max()), (tok, h)
+
+
+
 # ----------------------------------------------------------------------------------- invariants
 def pin_table_permutation_invariance():
     """Paged == contiguous: any placement of the pages gives bit-identical output."""
@@ -369,7 +399,7 @@ PINS = [pin_single_key_returns_its_value, pin_two_keys_logistic_weights,
         pin_table_permutation_invariance, pin_decode_equals_last_prefill_row,
         pin_chunked_equals_unchunked, pin_softmax_weights_and_convexity, pin_gqa_group_symmetry,
         pin_needle_visibility, pin_every_position_is_gathered_from_its_slot,
-        pin_append_writes_exactly_the_live_slots, pin_fig7_worked_example, pin_eq5_eq6_and_counters, pin_chunk_size_selection, pin_scaler_and_router]
+        pin_append_writes_exactly_the_live_slots, pin_selected_tokens_are_the_named_ones, pin_fig7_worked_example, pin_eq5_eq6_and_counters, pin_chunk_size_selection, pin_scaler_and_router]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=[p.__name__ for p in PINS])
@@ -391,6 +421,8 @@ MUTANTS = [
     ("append_slot_off", "int slot = t % P;", "int slot = (t + 1) % P;"),
     ("append_v_into_k", "memcpy(pool + pool_index(page, 1, g, slot, Hkv, P, D), vs", "memcpy(pool + pool_index(page, 0, g, slot, Hkv, P, D), vs"),
     ("dropped_d_term", "for (int d = 0; d < D; ++d) dot +=", "for (int d = 1; d < D; ++d) dot +="),
+    ("sel_output_slot", "out + ((size_t)o * Hq + h) * D, s);", "out + ((size_t)(sel ? n_out - 1 - o : o) * Hq + h) * D, s);"),
+    ("sel_ignored_in_worker", "long tok = sel ? sel[o] : o;\n      int r = tok_row[tok]", "long tok = o;\n      int r = tok_row[tok]"),
     ("pool_kv_stride", "((((size_t)page * 2 + (size_t)kv) * (size_t)Hkv + (size_t)head)", "((((size_t)page * 2 + (size_t)kv) * (size_t)Hkv + (size_t)(Hkv - 1 - head))"),
 ]
 
