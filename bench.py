@@ -40,6 +40,8 @@ WORKLOADS = {
     "config2": (wl.config2, "decode-only batch, 8B-shaped layer (64 decode rows, ctx lognormal median 2048)"),
     "config3": (wl.config3, "convertible-decoder burst, 8B-shaped layer (64 decode rows + one fresh 2048-token prefill chunk)"),
     "config4": (wl.config4, "chunked-prefill continuation, 8B-shaped layer (128 decode rows + 4 chunks of 512 tokens)"),
+    "prefill_8192_70b": (None, "one fresh 8192-token prefill chunk alone, 70B-shaped layer (the tile path by itself)"),
+    "prefill_2048_8b": (None, "one fresh 2048-token prefill chunk alone, 8B-shaped layer (config3's chunk by itself)"),
     "config5": (None, "bursty trace replay, 70B-shaped layer (200 steps, Gamma arrivals CV=4, <=256 decodes, one prefill task at a time)"),
     "config5_chunked": (None, "the same bursty trace under a chunk size of 2304 (2048 prefill tokens + 256 decode rows): "
                               "prompts continue over several steps, up to 4 requests' chunks share a step"),
@@ -208,6 +210,10 @@ def replay_heavy_batch():
 def make_static_batch(workload: str, rank: int):
     if workload in REPLAY_TRACE:
         return replay_heavy_batch()
+    if workload == "prefill_8192_70b":
+        return wl.make_batch(workload, wl.LLAMA70B, [0], [8192], seed=rank_seed(81, rank), chunk_size=8192)
+    if workload == "prefill_2048_8b":
+        return wl.make_batch(workload, wl.LLAMA8B, [0], [2048], seed=rank_seed(82, rank), chunk_size=2048)
     make = WORKLOADS[workload][0]
     return make(seed=rank_seed(make.__defaults__[0], rank))
 
@@ -384,7 +390,9 @@ def run_static(args, world, rank, local, barrier, workload=None, light=False):
 
     kv_tokens = int((batch.ctx_len + batch.q_len).sum())
     cfg = {"decode_rows": batch.decode_tokens, "prefill_tokens": batch.prefill_tokens, "kv_tokens": kv_tokens,
-           "l2": "inputs larger than L2 (KV working set %.2f GB)" % (kv_tokens * s.kv_bytes_per_token / 1e9),
+           "l2": ("inputs larger than L2 (KV working set %.2f GB)" if kv_tokens * s.kv_bytes_per_token > 126e6 else
+                  "KV working set %.3f GB fits in L2 and is not flushed: a tensor-bound diagnostic, no HBM claim")
+                 % (kv_tokens * s.kv_bytes_per_token / 1e9),
            "timing": f"median of {n_blocks} blocks of {K} steps, CUDA events around each block, "
                      f"timed region {region_s:.2f} s"}
     e2e = None
@@ -588,7 +596,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = cpu_baseline_leg(r["batch"] if r["batch"] is not None else make_static_batch(args.workload, 0))
     if rank == 0:
-        shape = wl.LLAMA70B if args.workload in REPLAY_TRACE else wl.LLAMA8B
+        shape = wl.LLAMA70B if args.workload in REPLAY_TRACE or args.workload.endswith("70b") else wl.LLAMA8B
         cfg = {"workload": args.workload, "description": WORKLOADS[args.workload][1], "n_q_heads": shape.Hq,
                "n_kv_heads": shape.Hkv, "head_dim": shape.D, "page_size": shape.P,
                "parallelism": f"replicas x{world}"}

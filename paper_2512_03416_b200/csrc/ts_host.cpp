@@ -146,6 +146,7 @@ struct ts_ctx {
   uint64_t host_steps = 0;
   bool cuda_ready = false;
   CUtensorMap kv_map;               // TMA view of the pool, box = K and V of one (page, head) half
+  CUtensorMap kv_tile_map;          // same view, box = K or V of one (page, head) half
   void* encode_fn = nullptr;        // cuTensorMapEncodeTiled
   int n_sms = 0;
   int n_prefill_items = 0;          // of the current plan
@@ -209,12 +210,16 @@ int make_kv_maps(ts_ctx* c) {
   const cuuint64_t dims[5] = {D, P, H, 2, (cuuint64_t)c->cfg.n_pages};
   const cuuint64_t strides[4] = {D * 2, P * D * 2, H * P * D * 2, 2 * H * P * D * 2};
   const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-  const cuuint32_t box[5] = {64, (cuuint32_t)P, 1, 2, 1};
-  const CUresult r = ((EncodeFn)c->encode_fn)(&c->kv_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, c->cfg.kv_pool,
-                                              dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return cuda_fail(c, cudaErrorInvalidValue);
+  // kv_map: K and V of one (page, head) half together, for the decode units; kv_tile_map: one
+  // operand only, for the K and V tiles of the prefill path
+  for (int both = 1; both >= 0; --both) {
+    const cuuint32_t box[5] = {64, (cuuint32_t)P, 1, (cuuint32_t)(both ? 2 : 1), 1};
+    const CUresult r = ((EncodeFn)c->encode_fn)(both ? &c->kv_map : &c->kv_tile_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                                                5, c->cfg.kv_pool, dims, strides, box, estr,
+                                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail(c, cudaErrorInvalidValue);
+  }
   return TS_OK;
 }
 
@@ -645,7 +650,7 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
         }
         if (pe) c->prof_mixed.back() = decode_launched;
         d.append_arrivals = n_ctas + ((c->cfg.debug_flags & TS_DEBUG_LOSE_APPEND_ARRIVAL) ? 1 : 0);
-        TS_CUDA(c, ts::launch_mixed(d, q_map, c->kv_map, n_ctas, p, stream));
+        TS_CUDA(c, ts::launch_mixed(d, q_map, c->kv_map, c->kv_tile_map, n_ctas, p, stream));
       } else {
         ts::StepDevice dp = d;
         dp.n_items = c->n_prefill_items;

@@ -94,9 +94,10 @@ cudaError_t launch_combine(const StepDevice& s, cudaStream_t stream);
 // kernel also appends the step's new K/V itself (no launch_kv_append before it). With
 // n_prefill_ctas == n_ctas the decode splits are left to launch_decode. When it runs the decode
 // splits it also merges them (no launch_combine needed).
-// q_map views q as (head_dim, G, KV head, token), box 64 x G x 1 x 128/G.
-cudaError_t launch_mixed(const StepDevice& s, const CUtensorMap& q_map, const CUtensorMap& kv_map, int n_ctas,
-                         int n_prefill_ctas, cudaStream_t stream);
+// q_map views q as (head_dim, G, KV head, token), box 64 x G x 1 x 128/G. kv_tile_map is the pool
+// view of kv_map with a box of one operand only (64 x 16 x 1 x 1 x 1): the prefill tiles' K/V copies.
+cudaError_t launch_mixed(const StepDevice& s, const CUtensorMap& q_map, const CUtensorMap& kv_map,
+                         const CUtensorMap& kv_tile_map, int n_ctas, int n_prefill_ctas, cudaStream_t stream);
 cudaError_t launch_decode(const StepDevice& s, const CUtensorMap& kv_map, int n_sms, cudaStream_t stream);
 
 // Programmatic dependent launch: every kernel of a step is launched with the attribute that lets

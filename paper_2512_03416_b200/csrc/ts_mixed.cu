@@ -11,21 +11,27 @@
 // x the G query heads of one KV head per tile) against all keys they may see, 128 keys per block.
 // Per tile and block:
 //     S = Q K^T   (tcgen05.mma, operands in 128B-swizzled shared memory, fp32 accumulator in TMEM)
-//     online softmax by one warpgroup, one query row per thread, the score row in registers
+//     online softmax by two warpgroups, two threads per query row, half a score row in registers each
 //     O += P V    (tcgen05.mma, P read from TMEM as bf16, V from shared memory, O accumulates in TMEM)
 // The two tiles share every K/V block (half the shared-memory fill per flop) and run out of phase:
-// while one tile's warpgroup is in its softmax, the tensor pipe works for the other tile.
-// TMEM (512 columns): S_A, S_B, O_A, O_B, 128 columns each; P overwrites the first 64 columns of
-// its S. Warp roles: warps 0-3 softmax/epilogue of tile A, warps 4-7 of tile B (thread = TMEM lane =
-// query row), warps 8-9 K loaders, warps 10-11 V loaders (16-byte cp.async through the block table
-// into the swizzled operand layout; the first K-loader thread also claims the work units), warp 12
-// MMA issuer and TMEM owner, warp 13 Q loader (TMA).
+// while one tile's warpgroups are in their softmax, the tensor pipe works for the other tile.
+// TMEM (512 columns): S_A, S_B, O_A, O_B, 128 columns each; the P of the keys in a 64-column half
+// of S overwrites the first 32 columns of that half.
+// Warp roles: warps 0-3 / 8-11 softmax and epilogue of tile A (keys 0-63 / 64-127 of each block,
+// head_dim columns 0-63 / 64-127 of O), warps 4-7 / 12-15 the same for tile B (thread = TMEM lane =
+// query row; a warp can only reach the 32 lanes its index modulo 4 selects, so a row is split by
+// columns). The two threads of a row agree on the row maximum through shared memory and a
+// 64-thread mbarrier per block. Two softmax warps per tile and SM sub-partition hide each
+// other's instruction latencies: one warp per row quarter left the tensor pipe idle more than
+// half of the time although no unit was saturated. Warp 16 K loader, warp 17 V loader (16-byte
+// cp.async through the block table into the swizzled operand layout; the K loader's first thread
+// also claims the work units), warp 18 MMA issuer and TMEM owner, warp 19 Q loader (TMA).
 // All barrier phases follow running block counters, so the roles flow from one work unit into the
 // next without a CTA-wide stop: the loaders run ahead into the next unit's K/V, its Q tiles land
 // as soon as the last Q K^T of the current unit has been issued, and its first Q K^T overlaps
 // the epilogue of the current unit.
 // The O rescale is lazy: a row's reference maximum only moves when a block's maximum exceeds it by
-// more than 2^8, so most blocks never touch O and take a single pass over their scores.
+// more than 2^8, so most blocks never touch O.
 // The kernel starts by appending the step's new K/V to the pages itself (every CTA a share of
 // the tokens, then a launch-wide counter barrier), which saves a launch in front of it.
 // Every wait is bounded; a wait that runs out raises TS_DEV_TIMEOUT and the CTA drains.
@@ -40,15 +46,18 @@
 namespace ts {
 namespace {
 
-constexpr int kPfThreads = 512;                 // 8 softmax warps + 4 loader warps + MMA warp (+ Q-loader warp, 2 idle)
-// Register split (setmaxnreg works on whole warpgroups, hence the three idle warps): the block is
-// launched with 128 registers per thread; the two softmax warpgroups grow to hold their score
-// row, the loader and MMA warpgroups shrink. 256 * 176 + 128 * 64 + 128 * 96 = 512 * 128.
-constexpr int kRegsSoftmax = 176, kRegsLoader = 64, kRegsMma = 96;
-static_assert(256 * kRegsSoftmax + 128 * kRegsLoader + 128 * kRegsMma <= 512 * 128,
+constexpr int kPfThreads = 640;                 // 16 softmax warps + K loader, V loader, MMA and Q-loader warps
+constexpr int kSoftmaxWarps = 16;
+// Register split (setmaxnreg works on whole warpgroups): the block is launched with 96 registers
+// per thread; the four softmax warpgroups grow to hold their half score row, the fifth warpgroup
+// (loaders, MMA issuer) shrinks. In a CTA that runs decode units first, the two warpgroups that run
+// them take the registers the other two softmax warpgroups do not need yet.
+constexpr int kRegsLaunch = 96, kRegsSoftmax = 104, kRegsAux = 64, kRegsDecode = 168, kRegsParked = 24;
+static_assert(4 * 128 * kRegsSoftmax + 128 * kRegsAux <= kPfThreads * kRegsLaunch,
               "register split exceeds the launch's total");
-constexpr int kLoaderThreads = 64;              // per operand (K or V)
-constexpr int kWarpLoader0 = 8, kWarpMma = 12, kWarpSched = 13;
+static_assert(2 * 128 * kRegsDecode + 2 * 128 * kRegsParked + 128 * kRegsAux <= kPfThreads * kRegsLaunch,
+              "register split of the decode phase exceeds the launch's total");
+constexpr int kWarpLoader0 = 16, kWarpMma = 18, kWarpSched = 19;
 constexpr int kBlockKeys = 128;
 constexpr int kD = 128;
 constexpr int kTileBytes = 128 * kD * 2;        // one 128 x 128 bf16 operand tile: 32 KB
@@ -72,14 +81,21 @@ enum {
   BAR_O_FULL = BAR_P_FULL + 2,            // [2] per tile
   BAR_O_EMPTY = BAR_O_FULL + 2,           // [2] per tile: the epilogue has read O out of TMEM
   BAR_Q_EMPTY = BAR_O_EMPTY + 2,          // the last Q K^T of a work unit has consumed the Q tiles
-  BAR_COUNT = BAR_Q_EMPTY + 1
+  BAR_PAIR = BAR_Q_EMPTY + 1,             // [8] per tile and row quarter: the two warps that share the rows
+  BAR_V_LANDED = BAR_PAIR + 8,            // [kVStages] the copies of a V tile are in shared memory
+  BAR_COUNT = BAR_V_LANDED + kVStages
 };
 // misc words: [0] TMEM base address, [1] failure flag, [2] work units published so far;
 // then a ring of the published units' records (8 words each)
 constexpr int kOffMisc = kOffBar + BAR_COUNT * 8;
 constexpr int kOffRing = kOffMisc + 16;
 constexpr int kSchedRing = 8;
-constexpr int kSmemBytes = kOffRing + kSchedRing * 32 + 1024;
+// row statistics the two threads of a query row exchange: [tile][half][row] floats
+constexpr int kOffXchg = kOffRing + kSchedRing * 32;
+constexpr int kSmemBytes = kOffXchg + 2 * 2 * 128 * 4;
+// The operand tiles need a 1024-byte-aligned base. The kernel has no static shared memory, so its
+// dynamic window starts on such a boundary; the kernel checks that and refuses to run otherwise
+// (there is no room left for alignment slack).
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory one CTA can opt into");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -145,18 +161,6 @@ __device__ __forceinline__ void tmem_ld32(float* v, uint32_t taddr) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
-  const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,"
-      "%28,%29,%30,%31,%32};\n" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-      "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
-      "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
-      "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -181,15 +185,6 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
 __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) |
          ((128u >> 4) << 24);
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-  // src_bytes == 0 writes 16 zero bytes and reads nothing
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
 template <int N>
 __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(N)); }
@@ -229,39 +224,55 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// One row of a score block: p_i = 2^(x_i), x_i = v_i * scale + neg_m, for the 128 scores in v,
-// written as bf16 pairs into TMEM columns [t_p, t_p + 64); returns the row sum of the unrounded
-// p_i and, in x_max, the largest x_i. The maximum rides along in the issue slots the
-// special-function unit leaves free, so the common case needs no separate pass for it.
-__device__ __forceinline__ float exp_store(const float (&v)[128], float scale, float neg_m, uint32_t t_p,
-                                           float& x_max) {
+// Half a row of a score block: p_i = 2^(v_i * scale + neg_m) for the 64 scores in v, written as
+// bf16 pairs into TMEM columns [t_p, t_p + 32); returns the sum of the unrounded p_i.
+__device__ __forceinline__ float exp_store(const float (&v)[64], float scale, float neg_m, uint32_t t_p) {
   const uint64_t scale2 = pack_f2(scale, scale), negm2 = pack_f2(neg_m, neg_m);
   uint64_t sum_a = pack_f2(0.f, 0.f), sum_b = sum_a;
-  float xm0 = -CUDART_INF_F, xm1 = xm0, xm2 = xm0, xm3 = xm0;
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
+  for (int c = 0; c < 2; ++c) {
     uint32_t pk[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
       const int e = c * 32 + 2 * i;
       float x0, x1;
       unpack_f2(fma2(pack_f2(v[e], v[e + 1]), scale2, negm2), x0, x1);
-      if ((i & 3) == 0) xm0 = max3(xm0, x0, x1);
-      else if ((i & 3) == 1) xm1 = max3(xm1, x0, x1);
-      else if ((i & 3) == 2) xm2 = max3(xm2, x0, x1);
-      else xm3 = max3(xm3, x0, x1);
       const float p0 = ex2(x0), p1 = ex2(x1);
       if (i & 1) sum_b = add2(sum_b, pack_f2(p0, p1)); else sum_a = add2(sum_a, pack_f2(p0, p1));
       pk[i] = pack2(p0, p1);
     }
     tmem_st16(t_p + c * 16, pk);
   }
-  x_max = fmaxf(fmaxf(xm0, xm1), fmaxf(xm2, xm3));
   float a0, a1;
   unpack_f2(add2(sum_a, sum_b), a0, a1);
   return a0 + a1;
 }
-
+// Largest of the 64 raw scores of a half row.
+__device__ __forceinline__ float max64(const float (&v)[64]) {
+  float m0 = max3(v[0], v[1], v[2]), m1 = max3(v[3], v[4], v[5]);
+  float m2 = max3(v[6], v[7], v[8]), m3 = max3(v[9], v[10], v[11]);
+#pragma unroll
+  for (int i = 12; i < 60; i += 8) {
+    m0 = max3(m0, v[i], v[i + 1]);
+    m1 = max3(m1, v[i + 2], v[i + 3]);
+    m2 = max3(m2, v[i + 4], v[i + 5]);
+    m3 = max3(m3, v[i + 6], v[i + 7]);
+  }
+  m0 = max3(m0, v[60], v[61]);
+  m1 = max3(m1, v[62], v[63]);
+  return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+__device__ __forceinline__ void tmem_ld16(float* v, uint32_t taddr) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 // One prefill work unit as its claimer publishes it in shared memory (8 words), and the shape
 // every role derives from it.
 struct UnitRec {
@@ -302,12 +313,17 @@ __device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 0;\n" ::: "m
 
 __global__ void __launch_bounds__(kPfThreads, 1)
 mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
-             const __grid_constant__ CUtensorMap kv_map, const int n_prefill_ctas) {
+             const __grid_constant__ CUtensorMap kv_map, const __grid_constant__ CUtensorMap kv_tile_map,
+             const int n_prefill_ctas) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem = smem_raw + (base - smem_u32(smem_raw));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   pdl_launch_dependents();
+  if (base != smem_u32(smem_raw)) {          // never expected, see kSmemBytes
+    if (tid == 0) atomicOr(s.status, TS_DEV_BAD_INDEX);
+    return;
+  }
   const uint32_t bar0 = base + kOffBar;
   auto bar = [&](int i) { return bar0 + (uint32_t)i * 8u; };
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
@@ -354,9 +370,8 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
       misc[2] = 0;
       for (int i = 0; i < BAR_COUNT; ++i) {
         const bool softmax_arrives = (i >= BAR_P_FULL && i < BAR_P_FULL + 2) || (i >= BAR_O_EMPTY && i < BAR_O_EMPTY + 2);
-        const bool loaders_arrive = (i >= BAR_K_FULL && i < BAR_K_FULL + kKStages) ||
-                                    (i >= BAR_V_FULL && i < BAR_V_FULL + kVStages);
-        mbar_init(bar(i), softmax_arrives ? 128 : loaders_arrive ? kLoaderThreads : 1);
+        const bool pair = i >= BAR_PAIR && i < BAR_PAIR + 8;
+        mbar_init(bar(i), softmax_arrives ? 256 : pair ? 64 : 1);
       }
       mbar_init_fence();
     }
@@ -377,9 +392,12 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
     cta_sync();
     tc_fence_after();
   };
-  // Decode-first CTAs: warps 0-7 run the CTA's decode units, the other warps wait for them.
-  auto decode_phase_idle = [&]() {
+  // The fifth warpgroup (loaders, MMA issuer, Q loader): gives registers to the softmax warpgroups
+  // and, in a decode-first CTA, waits while warps 0-7 run the CTA's decode units.
+  auto aux_setup = [&]() {
+    reg_dec<kRegsAux>();
     if (decode_first) cta_sync();
+    prefill_setup();
   };
 
   // ---------------------------------------------------------------- KV append (Sec. 2.1)
@@ -410,25 +428,49 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
     cta_sync();
   }
 
-  if (warp < 8) {
-    // ------------------------------------------ softmax + epilogue: thread = query row of tile x
-    reg_inc<kRegsSoftmax>();
+  if (warp < kSoftmaxWarps) {
+    // ------------------ softmax + epilogue: thread = half of a query row of tile x (64 of the 128
+    // keys of every block, 64 of the 128 head_dim columns of O)
     if (decode_first) {
-      dec::decode_units<128, 1, 3>(s, &kv_map, smem, base, (int)blockIdx.x - n_prefill_ctas,
-                                   (int)gridDim.x - n_prefill_ctas);
-      if (tid == 0) {          // this CTA's split partials are written: count it as done
-        __threadfence();
-        atomicAdd(s.pf_queue + 1, 1);
+      if (warp < 8) {
+        reg_inc<kRegsDecode>();       // waits until the parked warpgroups have given their registers up
+        dec::decode_units<128, 1, 3>(s, &kv_map, smem, base, (int)blockIdx.x - n_prefill_ctas,
+                                     (int)gridDim.x - n_prefill_ctas);
+        if (tid == 0) {          // this CTA's split partials are written: count it as done
+          __threadfence();
+          atomicAdd(s.pf_queue + 1, 1);
+        }
+        fence_proxy_async();     // the prefill phase reuses this shared memory through other proxies
+        reg_dec<kRegsSoftmax>();
+        cta_sync();
+      } else {
+        reg_dec<kRegsParked>();
+        cta_sync();
+        reg_inc<kRegsSoftmax>();
       }
-      fence_proxy_async();     // the prefill phase reuses this shared memory through other proxies
-      cta_sync();
+    } else {
+      reg_inc<kRegsSoftmax>();
     }
     prefill_setup();
     const uint32_t tmem = misc[0];
-    const int x = warp >> 2;
+    const int x = (warp >> 2) & 1;          // tile
+    const int hf = warp >> 3;               // which half of the keys / of the head_dim columns
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tS = tmem + x * 128 + lane_addr, tO = tmem + 256 + x * 128 + lane_addr;
+    const uint32_t tS = tmem + x * 128 + hf * 64 + lane_addr;         // my 64 score columns; P goes to the first 32
+    const uint32_t tO = tmem + 256 + x * 128 + hf * 64 + lane_addr;   // my 64 columns of O
+    // The two warps that share a quarter of a tile's rows meet on an mbarrier (a bounded wait, like
+    // every other one here) around each exchange through shared memory.
+    const int pair_bar = BAR_PAIR + x * 4 + (warp & 3);
+    int n_pair = 0;
+    auto pair_sync = [&]() {
+      mbar_arrive(bar(pair_bar));
+      wait(pair_bar, n_pair & 1);
+      ++n_pair;
+    };
+    float* xchg = reinterpret_cast<float*>(smem + kOffXchg) + x * 256;   // [half][row] of my tile
+    float* xchg_mine = xchg + hf * 128 + row;
+    const float* xchg_other = xchg + (hf ^ 1) * 128 + row;
     const float scale = s.scale_log2;
     int sx = 0;                 // blocks of this tile in earlier work units: barrier phases follow it
     for (int k = 0;; ++k) {
@@ -444,81 +486,75 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
       for (int j = 0; j < nbx; ++j) {
         wait(BAR_S_FULL + x, (sx + j) & 1);
         tc_fence_after();
-        // the whole score row lives in registers: one trip to TMEM per block
-        float v[128];
+        // my half of the score row lives in registers: one trip to TMEM per block
+        float v[64];
         tmem_ld32(&v[0], tS);
         tmem_ld32(&v[32], tS + 32);
-        tmem_ld32(&v[64], tS + 64);
-        tmem_ld32(&v[96], tS + 96);
         tmem_ld_wait();
-        const int nvalid = lim - j * kBlockKeys;               // keys of this block the row may see
-        if (__any_sync(0xffffffffu, nvalid < kBlockKeys)) {    // only the blocks on the diagonal
+        const int nvalid = lim - j * kBlockKeys - hf * 64;     // keys of my half the row may see
+        if (__any_sync(0xffffffffu, nvalid < 64)) {            // only the blocks on the diagonal
 #pragma unroll
-          for (int i = 0; i < 128; ++i)
+          for (int i = 0; i < 64; ++i)
             if (i >= nvalid) v[i] = -CUDART_INF_F;             // 2^(-inf) = 0 exactly
         }
-        // p = 2^(s*scale - m_ref) as bf16 over the first 64 columns of S (the scores are in
-        // registers), against the reference the row already has: the result is exact for any
-        // common reference, and p <= 2^threshold keeps the bf16 P and the fp32 sums comfortable.
-        // Only a row whose block maximum exceeds its reference by more than the threshold (always
-        // on a unit's first block, seldom afterwards) moves the reference, rescales O and redoes
-        // the block.
-        float x_max = CUDART_INF_F, ls = 0.f;
-        if (j > 0) ls = exp_store(v, scale, -m_ref, tS, x_max);
-        const bool move = x_max > kRescaleThreshold;
-        if (__any_sync(0xffffffffu, move)) {
-          float alpha = 1.f;
-          if (j == 0) {
-            // row maximum of the raw scores (the scale is positive, so it commutes with max)
-            float m0 = max3(v[0], v[1], v[2]), m1 = max3(v[3], v[4], v[5]);
-            float m2 = max3(v[6], v[7], v[8]), m3 = max3(v[9], v[10], v[11]);
-#pragma unroll
-            for (int i = 12; i < 124; i += 8) {
-              m0 = max3(m0, v[i], v[i + 1]);
-              m1 = max3(m1, v[i + 2], v[i + 3]);
-              m2 = max3(m2, v[i + 4], v[i + 5]);
-              m3 = max3(m3, v[i + 6], v[i + 7]);
-            }
-            m0 = max3(m0, v[124], v[125]);
-            m1 = max3(m1, v[126], v[127]);
-            m_ref = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * scale;
-          } else {
+        // The row maximum over both halves, exactly: each thread posts the maximum of its half and
+        // reads its partner's (the scale is positive, so it commutes with max). A row of the last,
+        // diagonal block may be masked completely; it keeps its reference (block 0 always holds
+        // key 0, which every row sees).
+        *xchg_mine = max64(v);
+        pair_sync();
+        const float m_blk = fmaxf(*xchg_mine, *xchg_other) * scale;
+        // p = 2^(s*scale - m_ref) as bf16 over the first 32 columns of my half of S (the scores are
+        // in registers). Any common reference is exact; p <= 2^threshold keeps the bf16 P and the
+        // fp32 sums comfortable, so the reference only moves (and O is only rescaled) when the
+        // block maximum exceeds it by more than the threshold. Both threads of a row see the
+        // same numbers and take the same decision.
+        if (j == 0) {
+          m_ref = m_blk;
+        } else {
+          const bool move = m_blk > m_ref + kRescaleThreshold;
+          if (__any_sync(0xffffffffu, move)) {
+            float alpha = 1.f;
             if (move) {
-              alpha = ex2(-x_max);                            // 2^(old reference - new reference)
-              m_ref += x_max;
+              alpha = ex2(m_ref - m_blk);
+              m_ref = m_blk;
               l *= alpha;
             }
             wait(BAR_O_FULL + x, (sx + j - 1) & 1);           // P V of block j-1 has landed in O
             tc_fence_after();
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
-              float ov[32];
-              tmem_ld32(ov, tO + c * 32);
+              float ov[16];
+              tmem_ld16(ov, tO + c * 16);
               tmem_ld_wait();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) ov[i] *= alpha;
-              tmem_st32(tO + c * 32, ov);
+              for (int i = 0; i < 16; ++i) ov[i] *= alpha;
+              tmem_st16(tO + c * 16, *reinterpret_cast<const uint32_t(*)[16]>(ov));
             }
           }
-          ls = exp_store(v, scale, -m_ref, tS, x_max);
         }
-        l += ls;
+        l += exp_store(v, scale, -m_ref, tS);
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(bar(BAR_P_FULL + x));
       }
       if (nbx > 0) {
-        // epilogue: O / l -> bf16 -> global
+        // epilogue: O / l -> bf16 -> global; l is the sum over both halves of the keys. (The last
+        // P V has been issued, so the partner has arrived for the last block and is done with
+        // that block's exchange slots.)
         wait(BAR_O_FULL + x, (sx + nbx - 1) & 1);
         tc_fence_after();
-        const float inv = 1.f / l;
-        uint16_t* orow = s.out + ((size_t)(tok0 + tok) * s.Hq + u.kv_head * G + row % G) * kD;
+        *xchg_mine = l;
+        pair_sync();
+        const float inv = 1.f / (l + *xchg_other);
+        pair_sync();                      // both have read: the slots may be written again
+        uint16_t* orow = s.out + ((size_t)(tok0 + tok) * s.Hq + u.kv_head * G + row % G) * kD + hf * 64;
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c) {
           float ov[32];
           tmem_ld32(ov, tO + c * 32);
           tmem_ld_wait();
-          if (c == 3) {
+          if (c == 1) {
             tc_fence_before();
             mbar_arrive(bar(BAR_O_EMPTY + x));   // O is in registers: the next unit may overwrite it
           }
@@ -539,9 +575,9 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
     }
     // -------------------------------------------------------------- merge of the decode splits
     // By now the decode CTAs are normally long done; once all of them have counted themselves,
-    // these eight warps of every CTA merge the split rows between them.
+    // the first eight warps of every CTA merge the split rows between them.
     const int n_decode_ctas = (int)gridDim.x - n_prefill_ctas;
-    if (s.n_combines > 0 && n_decode_ctas > 0) {
+    if (warp < 8 && s.n_combines > 0 && n_decode_ctas > 0) {
       if (tid == 0) {
         const volatile int32_t* done = s.pf_queue + 1;
         const long long t0 = clock64();
@@ -596,223 +632,220 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
         *reinterpret_cast<uint2*>(s.out + ((size_t)c.token * s.Hq + h) * kD + lane * 4) = o;
       }
     }
-  } else if (warp < kWarpLoader0 + 4) {
-    // ------------------------------------------------------------------ K/V loaders
-    // 64 threads per operand copy each 128-key tile with 16-byte cp.async straight into the
-    // 128-byte-swizzled operand layout. (TMA is not used for K/V: with 16-token pages every
-    // tensor copy is only 2 KB, and the copy engine's per-request cost would bound the kernel.)
-    // K and V are two independent pipelines. A tile is announced at the start of a later
-    // iteration of its own loader, before that iteration waits for a free stage, so the
-    // announcement depends only on the copy having landed.
-    reg_dec<kRegsLoader>();
-    decode_phase_idle();
-    prefill_setup();
-    const int kv = (warp - kWarpLoader0) >> 1;               // 0: K, 1: V
-    const int t = tid - 256 - kv * kLoaderThreads;           // 0..63 inside the group
-    const int col16 = t & 15, rb = t >> 4;                   // chunk col16 of rows rb + 4 h + 8 i
-    const int stages = kv ? kVStages : kKStages;
-    const int lag = stages - 1;                              // tiles in flight besides the announced one
-    const int full = kv ? BAR_V_FULL : BAR_K_FULL, empty = kv ? BAR_V_EMPTY : BAR_K_EMPTY;
-    const uint32_t tile0 = base + (kv ? kOffV : kOffK);
-    const size_t page_stride = (size_t)2 * s.Hkv * kPageSize * kD;
-    // The first K-loader thread takes work units off the global queue, one at a time and only
-    // when the K loaders are ready for it (they run a few key blocks ahead of the tensor pipe, which
-    // hides the round trip), and publishes each to the other roles through a small ring.
-    int fetched = 0;
-    auto fetch_one = [&]() {
-      const int w = atomicAdd(s.pf_queue, 1);
-      UnitRec r = {};
-      r.w = -1;
-      if (w < n_units) {
-        const WorkItem it = s.items[w / s.Hkv];
-        r.w = w;
-        r.table_slot = s.row_slot[it.row];
-        r.kv_head = w % s.Hkv;
-        r.q_begin = it.q_begin;
-        r.q_count = it.q_count;
-        r.ctx = it.k_end - it.q_begin - it.q_count;
-        r.tok0 = s.row_tok0[it.row];
-        if ((unsigned)r.table_slot >= (unsigned)s.max_requests) {
-          atomicOr(s.status, TS_DEV_BAD_INDEX);
-          r.w = -1;
+  } else {
+    // warps 16-19 are one warpgroup: they change their register count with one instruction
+    aux_setup();
+    if (warp < kWarpLoader0 + 2) {
+      // ------------------------------------------------------------------ K/V loaders
+      // One warp per operand. A 128-key tile is sixteen tensor copies of 2 KB (one page of one KV
+      // head, 64 head_dim columns each; the page id is a coordinate of the copy, so scattered pages
+      // cost nothing extra), issued by sixteen lanes at once and landing in the 128-byte-swizzled
+      // operand layout the MMA reads. K tiles complete their "full" barrier by transaction bytes.
+      // V tiles complete a "landed" barrier first: the warp then clears, in shared memory, the V
+      // rows of a ragged last page (slots past the last key may hold anything, and 0 * NaN would
+      // poison O; the same rows of K only produce scores that are masked) and announces the tile.
+      // The loaders run up to a ring of stages ahead of the tensor pipe.
+      const int kv = warp - kWarpLoader0;                      // 0: K, 1: V
+      const int stages = kv ? kVStages : kKStages;
+      const int lag = stages - 1;                              // V tiles in flight besides the announced one
+      const int full = kv ? BAR_V_FULL : BAR_K_FULL, empty = kv ? BAR_V_EMPTY : BAR_K_EMPTY;
+      const uint32_t tile0 = base + (kv ? kOffV : kOffK);
+      if (lane == 0) tma_prefetch_desc(&kv_tile_map);
+      // The K loader's first thread takes work units off the global queue, one at a time and only
+      // when the K loader is ready for it (it runs a few key blocks ahead of the tensor pipe, which
+      // hides the round trip), and publishes each to the other roles through a small ring.
+      int fetched = 0;
+      auto fetch_one = [&]() {
+        const int w = atomicAdd(s.pf_queue, 1);
+        UnitRec r = {};
+        r.w = -1;
+        if (w < n_units) {
+          const WorkItem it = s.items[w / s.Hkv];
+          r.w = w;
+          r.table_slot = s.row_slot[it.row];
+          r.kv_head = w % s.Hkv;
+          r.q_begin = it.q_begin;
+          r.q_count = it.q_count;
+          r.ctx = it.k_end - it.q_begin - it.q_count;
+          r.tok0 = s.row_tok0[it.row];
+          if ((unsigned)r.table_slot >= (unsigned)s.max_requests) {
+            atomicOr(s.status, TS_DEV_BAD_INDEX);
+            r.w = -1;
+          }
         }
-      }
-      const int e = (fetched & (kSchedRing - 1)) * 2;
-      ring[e].x = r.w; ring[e].y = r.table_slot; ring[e].z = r.kv_head; ring[e].w = r.q_begin;
-      ring[e + 1].x = r.q_count; ring[e + 1].y = r.ctx; ring[e + 1].z = r.tok0; ring[e + 1].w = 0;
-      __threadfence_block();
-      misc[2] = (uint32_t)++fetched;
-    };
-    int g0 = 0;                                              // key blocks of earlier work units
-    for (int k = 0;; ++k) {
-      if (kv == 0 && t == 0) fetch_one();
-      PfUnit u;
-      if (!get_work(k, u)) break;
-      const int32_t* table_row = s.table + (size_t)u.table_slot * s.max_pages_per_req;
-      const size_t head_off = ((size_t)kv * s.Hkv + u.kv_head) * kPageSize * kD + col16 * 8;
-      auto fetch_pages = [&](int j, int (&pg)[8]) {
-#pragma unroll
-        for (int p = 0; p < 8; ++p) {
-          const int key = j * kBlockKeys + p * kPageSize;
-          int page = -1;
-          if (key < u.k_end) {
+        const int e = (fetched & (kSchedRing - 1)) * 2;
+        ring[e].x = r.w; ring[e].y = r.table_slot; ring[e].z = r.kv_head; ring[e].w = r.q_begin;
+        ring[e + 1].x = r.q_count; ring[e + 1].y = r.ctx; ring[e + 1].z = r.tok0; ring[e + 1].w = 0;
+        __threadfence_block();
+        misc[2] = (uint32_t)++fetched;
+      };
+      int g0 = 0;                                              // key blocks of earlier work units
+      for (int k = 0;; ++k) {
+        if (kv == 0 && lane == 0) fetch_one();
+        __syncwarp();
+        PfUnit u;
+        if (!get_work(k, u)) break;
+        const int32_t* table_row = s.table + (size_t)u.table_slot * s.max_pages_per_req;
+        // lane i < 16 copies page i / 2 of the tile, head_dim columns [64 (i % 2), +64)
+        auto fetch_page = [&](int j) {
+          const int key = j * kBlockKeys + (lane >> 1) * kPageSize;
+          int page = s.n_pages;                                // out of range on purpose: the copy delivers zeros
+          if (lane < 16 && key < u.k_end) {
             page = table_row[key >> 4];
             if ((unsigned)page >= (unsigned)s.n_pages) {
               atomicOr(s.status, TS_DEV_BAD_PAGE);
-              page = -1;
+              page = s.n_pages;
             }
           }
-          pg[p] = page;
-        }
-      };
-      auto announce = [&](int tile, int pending_allowed) {   // tile = block index within the unit
-        if (pending_allowed >= 1) cp_async_wait<1>(); else cp_async_wait<0>();
-        fence_proxy_async();
-        mbar_arrive(bar(full + (g0 + tile) % stages));
-      };
-      int pg[8];
-      fetch_pages(0, pg);
-      for (int j = 0; j < u.nb; ++j) {
-        const int g = g0 + j;
-        const int st = g % stages;
-        const int key0 = j * kBlockKeys;
-        if (j >= lag) announce(j - lag, lag - 1);              // V: tile j-2 (j-1 in flight); K: tile j-1
-        int pg_next[8];
-        if (j + 1 < u.nb) fetch_pages(j + 1, pg_next);         // table loads fly while this tile is issued
-        if (g >= stages) wait(empty + st, ((g / stages) & 1) ^ 1);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int r0 = rb + 4 * h;
-          const uint32_t dst = tile0 + st * kTileBytes +
-                               (uint32_t)((col16 >> 3) * kHalfBytes + r0 * 128 + (((col16 & 7) ^ r0) << 4));
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int rowk = r0 + 8 * i;
-            const int page = pg[i >> 1];
-            const bool valid = page >= 0 && key0 + rowk < u.k_end;   // rows past the last key are zero-filled
-            const uint16_t* src = valid ? s.pool + (size_t)page * page_stride + head_off + (rowk & 15) * kD : s.pool;
-            cp_async16(dst + i * 1024, src, valid ? 16 : 0);
+          return page;
+        };
+        auto announce = [&](int tile) {                        // V only; tile = block index within the unit
+          const int gt = g0 + tile, st = gt % stages;
+          wait(BAR_V_LANDED + st, (gt / stages) & 1);
+          const int first_bad = u.k_end - tile * kBlockKeys;   // rows from here on hold no key of the unit
+          if (first_bad < kBlockKeys && (first_bad & 15)) {
+            const int n_rows = 16 - (first_bad & 15);          // up to the end of that page; later pages were not copied
+            unsigned char* vt = smem + kOffV + st * kTileBytes;
+            for (int i = lane; i < n_rows * 16; i += 32) {
+              const int r = first_bad + (i >> 4), c = i & 15;  // a row is 8 chunks of 16 bytes in each 64-column half
+              *reinterpret_cast<uint4*>(vt + (c >> 3) * kHalfBytes + r * 128 + ((c & 7) << 4)) = make_uint4(0, 0, 0, 0);
+            }
+            fence_proxy_async();
           }
-        }
-        cp_async_commit();
-#pragma unroll
-        for (int p = 0; p < 8; ++p) pg[p] = pg_next[p];
-      }
-      // the last `lag` tiles (fewer when the unit is short) have not been announced yet
-      for (int tile = max(0, u.nb - lag); tile < u.nb; ++tile) announce(tile, u.nb - 1 - tile);
-      g0 += u.nb;
-    }
-  } else {
-    // ------------------------------------------------------------------- MMA issuer
-    reg_dec<kRegsMma>();          // warps 14-15 only complete the fourth warpgroup
-    decode_phase_idle();
-    prefill_setup();
-    if (warp == kWarpMma) {
-      const uint32_t tmem = misc[0];
-      const uint32_t issue = elect_one();
-      // the warp keeps its own failure flag in a register: nothing on its path reads shared memory
-      bool dead = false;
-      auto iwait = [&](int i, uint32_t parity) {
-        if (!mbar_wait(bar(i), parity, dead ? 2000 : s.wait_cycles)) {
-          dead = true;
-          give_up();
-        }
-      };
-      constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
-      // descriptors differ only in their start-address field (16-byte units in the low bits)
-      const uint64_t q_desc0 = smem_desc(base + kOffQ, 0, 1024);
-      const uint64_t k_desc0 = smem_desc(base + kOffK, 0, 1024);
-      const uint64_t v_desc0 = smem_desc(base + kOffV, kHalfBytes, 1024);
-      auto issue_qk = [&](int x, int g) {          // S_x = Q_x K(g)^T
-        const uint64_t q_desc = q_desc0 + (uint64_t)((x * kTileBytes) >> 4);
-        const uint64_t k_desc = k_desc0 + (uint64_t)(((g % kKStages) * kTileBytes) >> 4);
-#pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks) {
-          const uint64_t off = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
-          mma_ss(tmem + x * 128, q_desc + off, k_desc + off, idesc_qk, ks > 0, issue);
-        }
-        tc_commit(bar(BAR_S_FULL + x), issue);
-      };
-      auto issue_pv = [&](int x, int g, bool first) {   // O_x (+)= P_x V(g)
-        const uint64_t v_desc = v_desc0 + (uint64_t)(((g % kVStages) * kTileBytes) >> 4);
-#pragma unroll
-        for (int kk = 0; kk < kBlockKeys / 16; ++kk)
-          mma_ts(tmem + 256 + x * 128, tmem + x * 128 + kk * 8, v_desc + (uint64_t)((kk * 2048) >> 4), idesc_pv,
-                 (!first || kk > 0) ? 1u : 0u, issue);
-        tc_commit(bar(BAR_O_FULL + x), issue);
-      };
-      int g0 = 0;                 // key blocks of earlier work units (K/V ring position)
-      int sxb[2] = {0, 0};        // blocks per tile in earlier work units (S/P/O phases)
-      int used[2] = {0, 0};       // earlier work units in which the tile had rows (O_EMPTY phases)
-      for (int k = 0;; ++k) {
-        PfUnit u;
-        if (!get_work(k, u)) break;
-        // Order: both Q K^T of block 0; then per block, for tile A then tile B:
-        // P V of block j followed at once by Q K^T of block j+1 of the same tile, so that the
-        // tile's warpgroup gets its next scores while the pipe turns to the other tile.
-        iwait(BAR_Q, k & 1);
-        iwait(BAR_K_FULL + g0 % kKStages, (g0 / kKStages) & 1);
-        tc_fence_after();
-        if (!dead) {
-          if (u.nb_a > 0) issue_qk(0, g0);
-          if (u.nb_b > 0) issue_qk(1, g0);
-          tc_commit(bar(BAR_K_EMPTY + g0 % kKStages), issue);
-          if (u.nb == 1) tc_commit(bar(BAR_Q_EMPTY), issue);
-        }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(full + st));
+        };
+        int page = fetch_page(0);
         for (int j = 0; j < u.nb; ++j) {
           const int g = g0 + j;
-          const bool next = j + 1 < u.nb;
+          const int st = g % stages;
+          if (kv && j >= lag) announce(j - lag);
+          const int page_next = j + 1 < u.nb ? fetch_page(j + 1) : 0;   // the table load flies while this tile is issued
+          if (g >= stages) wait(empty + st, ((g / stages) & 1) ^ 1);
+          const uint32_t landed = bar(kv ? BAR_V_LANDED + st : full + st);
+          if (misc[1] == 0) {                                  // after a failure no new copies are started
+            if (lane == 0) mbar_expect_tx(landed, kTileBytes);
+            __syncwarp();
+            if (lane < 16)
+              tma_load_5d(tile0 + st * kTileBytes + (lane & 1) * kHalfBytes + (lane >> 1) * 2048, &kv_tile_map, landed,
+                          (lane & 1) * 64, 0, u.kv_head, kv, page);
+          }
+          page = page_next;
+        }
+        // the last `lag` V tiles (fewer when the unit is short) have not been announced yet
+        if (kv)
+          for (int tile = max(0, u.nb - lag); tile < u.nb; ++tile) announce(tile);
+        g0 += u.nb;
+      }
+    } else {
+      // ------------------------------------------------------------------- MMA issuer
+      if (warp == kWarpMma) {
+        const uint32_t tmem = misc[0];
+        const uint32_t issue = elect_one();
+        // the warp keeps its own failure flag in a register: nothing on its path reads shared memory
+        bool dead = false;
+        auto iwait = [&](int i, uint32_t parity) {
+          if (!mbar_wait(bar(i), parity, dead ? 2000 : s.wait_cycles)) {
+            dead = true;
+            give_up();
+          }
+        };
+        constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
+        // descriptors differ only in their start-address field (16-byte units in the low bits)
+        const uint64_t q_desc0 = smem_desc(base + kOffQ, 0, 1024);
+        const uint64_t k_desc0 = smem_desc(base + kOffK, 0, 1024);
+        const uint64_t v_desc0 = smem_desc(base + kOffV, kHalfBytes, 1024);
+        auto issue_qk = [&](int x, int g) {          // S_x = Q_x K(g)^T
+          const uint64_t q_desc = q_desc0 + (uint64_t)((x * kTileBytes) >> 4);
+          const uint64_t k_desc = k_desc0 + (uint64_t)(((g % kKStages) * kTileBytes) >> 4);
 #pragma unroll
-          for (int x = 0; x < 2; ++x) {
-            const int nbx = x ? u.nb_b : u.nb_a;
-            if (j < nbx) {
-              iwait(BAR_P_FULL + x, (sxb[x] + j) & 1);
-              if (x == 0 || j >= u.nb_a) iwait(BAR_V_FULL + g % kVStages, (g / kVStages) & 1);
-              if (j == 0 && used[x] > 0) iwait(BAR_O_EMPTY + x, (used[x] - 1) & 1);   // the previous unit's O has been read
-              tc_fence_after();
-              if (!dead) issue_pv(x, g, j == 0);
-            }
-            if (x == 1 && !dead) tc_commit(bar(BAR_V_EMPTY + g % kVStages), issue);   // both tiles are done with V(g)
-            if (next) {
-              if (x == 0 || j + 1 >= u.nb_a) iwait(BAR_K_FULL + (g + 1) % kKStages, ((g + 1) / kKStages) & 1);
-              tc_fence_after();
-              if (j + 1 < nbx && !dead) issue_qk(x, g + 1);
-              if (x == 1 && !dead) {
-                tc_commit(bar(BAR_K_EMPTY + (g + 1) % kKStages), issue);
-                if (j + 2 == u.nb) tc_commit(bar(BAR_Q_EMPTY), issue);   // that was the unit's last Q K^T
+          for (int ks = 0; ks < kD / 16; ++ks) {
+            const uint64_t off = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+            mma_ss(tmem + x * 128, q_desc + off, k_desc + off, idesc_qk, ks > 0, issue);
+          }
+          tc_commit(bar(BAR_S_FULL + x), issue);
+        };
+        auto issue_pv = [&](int x, int g, bool first) {   // O_x (+)= P_x V(g)
+          const uint64_t v_desc = v_desc0 + (uint64_t)(((g % kVStages) * kTileBytes) >> 4);
+#pragma unroll
+          for (int kk = 0; kk < kBlockKeys / 16; ++kk)   // P of keys 0-63 sits in columns 0-31 of S, of keys 64-127 in 64-95
+            mma_ts(tmem + 256 + x * 128, tmem + x * 128 + (kk >> 2) * 64 + (kk & 3) * 8,
+                   v_desc + (uint64_t)((kk * 2048) >> 4), idesc_pv, (!first || kk > 0) ? 1u : 0u, issue);
+          tc_commit(bar(BAR_O_FULL + x), issue);
+        };
+        int g0 = 0;                 // key blocks of earlier work units (K/V ring position)
+        int sxb[2] = {0, 0};        // blocks per tile in earlier work units (S/P/O phases)
+        int used[2] = {0, 0};       // earlier work units in which the tile had rows (O_EMPTY phases)
+        for (int k = 0;; ++k) {
+          PfUnit u;
+          if (!get_work(k, u)) break;
+          // Order: both Q K^T of block 0; then per block, for tile A then tile B:
+          // P V of block j followed at once by Q K^T of block j+1 of the same tile, so that the
+          // tile's warpgroup gets its next scores while the pipe turns to the other tile.
+          iwait(BAR_Q, k & 1);
+          iwait(BAR_K_FULL + g0 % kKStages, (g0 / kKStages) & 1);
+          tc_fence_after();
+          if (!dead) {
+            if (u.nb_a > 0) issue_qk(0, g0);
+            if (u.nb_b > 0) issue_qk(1, g0);
+            tc_commit(bar(BAR_K_EMPTY + g0 % kKStages), issue);
+            if (u.nb == 1) tc_commit(bar(BAR_Q_EMPTY), issue);
+          }
+          for (int j = 0; j < u.nb; ++j) {
+            const int g = g0 + j;
+            const bool next = j + 1 < u.nb;
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+              const int nbx = x ? u.nb_b : u.nb_a;
+              if (j < nbx) {
+                iwait(BAR_P_FULL + x, (sxb[x] + j) & 1);
+                if (x == 0 || j >= u.nb_a) iwait(BAR_V_FULL + g % kVStages, (g / kVStages) & 1);
+                if (j == 0 && used[x] > 0) iwait(BAR_O_EMPTY + x, (used[x] - 1) & 1);   // the previous unit's O has been read
+                tc_fence_after();
+                if (!dead) issue_pv(x, g, j == 0);
+              }
+              if (x == 1 && !dead) tc_commit(bar(BAR_V_EMPTY + g % kVStages), issue);   // both tiles are done with V(g)
+              if (next) {
+                if (x == 0 || j + 1 >= u.nb_a) iwait(BAR_K_FULL + (g + 1) % kKStages, ((g + 1) / kKStages) & 1);
+                tc_fence_after();
+                if (j + 1 < nbx && !dead) issue_qk(x, g + 1);
+                if (x == 1 && !dead) {
+                  tc_commit(bar(BAR_K_EMPTY + (g + 1) % kKStages), issue);
+                  if (j + 2 == u.nb) tc_commit(bar(BAR_Q_EMPTY), issue);   // that was the unit's last Q K^T
+                }
               }
             }
           }
-        }
-        g0 += u.nb;
+          g0 += u.nb;
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          const int nbx = x ? u.nb_b : u.nb_a;
-          sxb[x] += nbx;
-          used[x] += nbx > 0;
+          for (int x = 0; x < 2; ++x) {
+            const int nbx = x ? u.nb_b : u.nb_a;
+            sxb[x] += nbx;
+            used[x] += nbx > 0;
+          }
         }
       }
-    }
-    if (warp == kWarpSched && lane == 0) {
-      // ------------------------------------------------------------------ Q loader
-      // Brings in each work unit's Q tiles by TMA once the previous unit's last Q K^T is done.
-      tma_prefetch_desc(&q_map);
-      for (int k = 0;; ++k) {
-        PfUnit u;
-        if (!get_work(k, u)) break;
-        const int ta = u.tok0 + u.q_begin;
-        if (k > 0) wait(BAR_Q_EMPTY, (k - 1) & 1);
-        // a box delivers 64 columns of tile_tokens * G packed rows (all 128 only when G divides 128)
-        mbar_expect_tx(bar(BAR_Q), (u.cnt_b > 0 ? 2 : 1) * 2 * (tile_tokens * G * 128));
-        tma_load_4d(base + kOffQ, &q_map, bar(BAR_Q), 0, 0, u.kv_head, ta);
-        tma_load_4d(base + kOffQ + kHalfBytes, &q_map, bar(BAR_Q), 64, 0, u.kv_head, ta);
-        if (u.cnt_b > 0) {
-          tma_load_4d(base + kOffQ + kTileBytes, &q_map, bar(BAR_Q), 0, 0, u.kv_head, ta + tile_tokens);
-          tma_load_4d(base + kOffQ + kTileBytes + kHalfBytes, &q_map, bar(BAR_Q), 64, 0, u.kv_head, ta + tile_tokens);
+      if (warp == kWarpSched && lane == 0) {
+        // ------------------------------------------------------------------ Q loader
+        // Brings in each work unit's Q tiles by TMA once the previous unit's last Q K^T is done.
+        tma_prefetch_desc(&q_map);
+        for (int k = 0;; ++k) {
+          PfUnit u;
+          if (!get_work(k, u)) break;
+          const int ta = u.tok0 + u.q_begin;
+          if (k > 0) wait(BAR_Q_EMPTY, (k - 1) & 1);
+          // a box delivers 64 columns of tile_tokens * G packed rows (all 128 only when G divides 128)
+          mbar_expect_tx(bar(BAR_Q), (u.cnt_b > 0 ? 2 : 1) * 2 * (tile_tokens * G * 128));
+          tma_load_4d(base + kOffQ, &q_map, bar(BAR_Q), 0, 0, u.kv_head, ta);
+          tma_load_4d(base + kOffQ + kHalfBytes, &q_map, bar(BAR_Q), 64, 0, u.kv_head, ta);
+          if (u.cnt_b > 0) {
+            tma_load_4d(base + kOffQ + kTileBytes, &q_map, bar(BAR_Q), 0, 0, u.kv_head, ta + tile_tokens);
+            tma_load_4d(base + kOffQ + kTileBytes + kHalfBytes, &q_map, bar(BAR_Q), 64, 0, u.kv_head, ta + tile_tokens);
+          }
         }
       }
+      __syncwarp();
     }
-    __syncwarp();
   }
   tc_fence_before();
   cta_sync();
@@ -831,8 +864,8 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
 
 }  // namespace
 
-cudaError_t launch_mixed(const StepDevice& s, const CUtensorMap& q_map, const CUtensorMap& kv_map, int n_ctas,
-                         int n_prefill_ctas, cudaStream_t stream) {
+cudaError_t launch_mixed(const StepDevice& s, const CUtensorMap& q_map, const CUtensorMap& kv_map,
+                         const CUtensorMap& kv_tile_map, int n_ctas, int n_prefill_ctas, cudaStream_t stream) {
   if (s.n_prefill_items <= 0 || n_ctas <= 0) return cudaSuccess;
   const int G = s.Hq / s.Hkv;
   size_t smem = kSmemBytes;
@@ -842,7 +875,7 @@ cudaError_t launch_mixed(const StepDevice& s, const CUtensorMap& q_map, const CU
   }
   cudaError_t e = cudaFuncSetAttribute(mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  return launch_pdl(mixed_kernel, dim3(n_ctas), dim3(kPfThreads), smem, stream, s, q_map, kv_map, n_prefill_ctas);
+  return launch_pdl(mixed_kernel, dim3(n_ctas), dim3(kPfThreads), smem, stream, s, q_map, kv_map, kv_tile_map, n_prefill_ctas);
 }
 
 }  // namespace ts
