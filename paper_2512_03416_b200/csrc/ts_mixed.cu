@@ -224,11 +224,13 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Half a row of a score block: p_i = 2^(v_i * scale + neg_m) for the 64 scores in v, written as
-// bf16 pairs into TMEM columns [t_p, t_p + 32); returns the sum of the unrounded p_i.
-__device__ __forceinline__ float exp_store(const float (&v)[64], float scale, float neg_m, uint32_t t_p) {
+// Half a row of a score block: p_i = 2^(x_i), x_i = v_i * scale + neg_m, for the 64 scores in v,
+// written as bf16 pairs into TMEM columns [t_p, t_p + 32); returns the sum of the unrounded p_i
+// and, in x_max, the largest x_i (it rides along in issue slots the exponentials leave free).
+__device__ __forceinline__ float exp_store(const float (&v)[64], float scale, float neg_m, uint32_t t_p, float& x_max) {
   const uint64_t scale2 = pack_f2(scale, scale), negm2 = pack_f2(neg_m, neg_m);
   uint64_t sum_a = pack_f2(0.f, 0.f), sum_b = sum_a;
+  float xm0 = -CUDART_INF_F, xm1 = xm0;
 #pragma unroll
   for (int c = 0; c < 2; ++c) {
     uint32_t pk[16];
@@ -237,12 +239,14 @@ __device__ __forceinline__ float exp_store(const float (&v)[64], float scale, fl
       const int e = c * 32 + 2 * i;
       float x0, x1;
       unpack_f2(fma2(pack_f2(v[e], v[e + 1]), scale2, negm2), x0, x1);
+      if (i & 1) xm1 = max3(xm1, x0, x1); else xm0 = max3(xm0, x0, x1);
       const float p0 = ex2(x0), p1 = ex2(x1);
       if (i & 1) sum_b = add2(sum_b, pack_f2(p0, p1)); else sum_a = add2(sum_a, pack_f2(p0, p1));
       pk[i] = pack2(p0, p1);
     }
     tmem_st16(t_p + c * 16, pk);
   }
+  x_max = fmaxf(xm0, xm1);
   float a0, a1;
   unpack_f2(add2(sum_a, sum_b), a0, a1);
   return a0 + a1;
@@ -463,10 +467,14 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
     // every other one here) around each exchange through shared memory.
     const int pair_bar = BAR_PAIR + x * 4 + (warp & 3);
     int n_pair = 0;
-    auto pair_sync = [&]() {
-      mbar_arrive(bar(pair_bar));
+    auto pair_arrive = [&]() { mbar_arrive(bar(pair_bar)); };
+    auto pair_wait = [&]() {
       wait(pair_bar, n_pair & 1);
       ++n_pair;
+    };
+    auto pair_sync = [&]() {
+      pair_arrive();
+      pair_wait();
     };
     float* xchg = reinterpret_cast<float*>(smem + kOffXchg) + x * 256;   // [half][row] of my tile
     float* xchg_mine = xchg + hf * 128 + row;
@@ -501,19 +509,28 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
         // reads its partner's (the scale is positive, so it commutes with max). A row of the last,
         // diagonal block may be masked completely; it keeps its reference (block 0 always holds
         // key 0, which every row sees).
-        *xchg_mine = max64(v);
-        pair_sync();
-        const float m_blk = fmaxf(*xchg_mine, *xchg_other) * scale;
         // p = 2^(s*scale - m_ref) as bf16 over the first 32 columns of my half of S (the scores are
         // in registers). Any common reference is exact; p <= 2^threshold keeps the bf16 P and the
         // fp32 sums comfortable, so the reference only moves (and O is only rescaled) when the
         // block maximum exceeds it by more than the threshold. Both threads of a row see the
-        // same numbers and take the same decision.
+        // same numbers and take the same decision. After the first block of a unit the
+        // exponentials are taken at once against the reference the row already has, and the
+        // maximum rides along with them: that is nearly always the final answer, and a warp with
+        // a row that does move simply takes them again.
+        float ls = 0.f, x_max;
         if (j == 0) {
-          m_ref = m_blk;
+          *xchg_mine = max64(v) * scale;                       // first block of a unit: the maximum itself
         } else {
-          const bool move = m_blk > m_ref + kRescaleThreshold;
-          if (__any_sync(0xffffffffu, move)) {
+          ls = exp_store(v, scale, -m_ref, tS, x_max);
+          *xchg_mine = x_max + m_ref;                          // largest s*scale of my half
+        }
+        pair_sync();
+        const float m_blk = fmaxf(*xchg_mine, *xchg_other);
+        const bool move = j == 0 || m_blk > m_ref + kRescaleThreshold;
+        if (__any_sync(0xffffffffu, move)) {
+          if (j == 0) {
+            m_ref = m_blk;
+          } else {
             float alpha = 1.f;
             if (move) {
               alpha = ex2(m_ref - m_blk);
@@ -532,8 +549,9 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
               tmem_st16(tO + c * 16, *reinterpret_cast<const uint32_t(*)[16]>(ov));
             }
           }
+          ls = exp_store(v, scale, -m_ref, tS, x_max);
         }
-        l += exp_store(v, scale, -m_ref, tS);
+        l += ls;
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(bar(BAR_P_FULL + x));
@@ -744,8 +762,10 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
         const uint32_t issue = elect_one();
         // the warp keeps its own failure flag in a register: nothing on its path reads shared memory
         bool dead = false;
+        // The issuer polls its barriers instead of parking on them: it is the only warp that does,
+        // and every cycle between a tile's P and its next scores is on the critical path.
         auto iwait = [&](int i, uint32_t parity) {
-          if (!mbar_wait(bar(i), parity, dead ? 2000 : s.wait_cycles)) {
+          if (!mbar_poll(bar(i), parity, dead ? 2000 : s.wait_cycles)) {
             dead = true;
             give_up();
           }
