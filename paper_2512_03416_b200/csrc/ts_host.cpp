@@ -517,8 +517,8 @@ bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 // How many CTAs of the mixed kernel take prefill tiles only, the rest streaming the decode rows
 // first and joining the prefill queue afterwards. Cost model in SM-microseconds, calibrated on a
-// B200: next to streaming decode CTAs a prefill work unit costs ~3.4 us per 128-key block pair
-// plus ~3 us; the decode rows move their K/V at a fraction of the full-chip rate that falls off as
+// B200: next to streaming decode CTAs a prefill work unit costs ~2.1 us per 128-key block pair
+// plus ~2 us; the decode rows move their K/V at a fraction of the full-chip rate that falls off as
 // fewer SMs pull on HBM, faster with eight query heads per KV head (twice the arithmetic per page)
 // than with four.
 //   G <= 4: an SM streams a decode unit at 70 GB/s plus ~2 us per unit, and all of them together
@@ -531,7 +531,7 @@ int choose_prefill_ctas(const ts_ctx* c, int n_ctas, double prefill_block_pairs,
   static const double kSm8[] = {0, 48, 64, 74, 84, 100, 116, 132, 148};
   static const double kRate8[] = {0, 0.475, 0.62, 0.715, 0.78, 0.85, 0.92, 0.95, 1.0};
   const bool wide = c->G > 4;
-  const double w_pf = prefill_block_pairs * 3.4 + prefill_units * 3.0;
+  const double w_pf = prefill_block_pairs * 2.1 + prefill_units * 2.0;
   const double t_dec_full = decode_bytes / 6.1e6;   // us at 6.1 TB/s
   const double unit_bytes = decode_bytes / std::max(1.0, decode_units);
   const double sm_rate = unit_bytes / (unit_bytes / 70e3 + 2.0);   // bytes per us and SM

@@ -225,26 +225,22 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 }
 
 // Half a row of a score block: p_i = 2^(x_i), x_i = v_i * scale + neg_m, for the 64 scores in v,
-// written as bf16 pairs into TMEM columns [t_p, t_p + 32); returns the sum of the unrounded p_i
-// and, in x_max, the largest x_i (it rides along in issue slots the exponentials leave free).
-__device__ __forceinline__ float exp_store(const float (&v)[64], float scale, float neg_m, uint32_t t_p, float& x_max) {
+// as bf16 pairs in pk (the scores are not needed afterwards, so their registers come free as
+// the loop advances); returns the sum of the unrounded p_i and, in x_max, the largest x_i (it
+// rides along in issue slots the exponentials leave free).
+__device__ __forceinline__ float exp_pack(const float (&v)[64], float scale, float neg_m, uint32_t (&pk)[32], float& x_max) {
   const uint64_t scale2 = pack_f2(scale, scale), negm2 = pack_f2(neg_m, neg_m);
   uint64_t sum_a = pack_f2(0.f, 0.f), sum_b = sum_a;
   float xm0 = -CUDART_INF_F, xm1 = xm0;
 #pragma unroll
-  for (int c = 0; c < 2; ++c) {
-    uint32_t pk[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const int e = c * 32 + 2 * i;
-      float x0, x1;
-      unpack_f2(fma2(pack_f2(v[e], v[e + 1]), scale2, negm2), x0, x1);
-      if (i & 1) xm1 = max3(xm1, x0, x1); else xm0 = max3(xm0, x0, x1);
-      const float p0 = ex2(x0), p1 = ex2(x1);
-      if (i & 1) sum_b = add2(sum_b, pack_f2(p0, p1)); else sum_a = add2(sum_a, pack_f2(p0, p1));
-      pk[i] = pack2(p0, p1);
-    }
-    tmem_st16(t_p + c * 16, pk);
+  for (int i = 0; i < 32; ++i) {
+    float x0, x1, p0, p1;
+    unpack_f2(fma2(pack_f2(v[2 * i], v[2 * i + 1]), scale2, negm2), x0, x1);
+    if (i & 1) xm1 = max3(xm1, x0, x1); else xm0 = max3(xm0, x0, x1);
+    p0 = ex2(x0);
+    p1 = ex2(x1);
+    if (i & 1) sum_b = add2(sum_b, pack_f2(p0, p1)); else sum_a = add2(sum_a, pack_f2(p0, p1));
+    pk[i] = pack2(p0, p1);
   }
   x_max = fmaxf(xm0, xm1);
   float a0, a1;
@@ -494,43 +490,46 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
       for (int j = 0; j < nbx; ++j) {
         wait(BAR_S_FULL + x, (sx + j) & 1);
         tc_fence_after();
-        // my half of the score row lives in registers: one trip to TMEM per block
+        // my half of the score row comes into registers: one trip to TMEM per block
         float v[64];
-        tmem_ld32(&v[0], tS);
-        tmem_ld32(&v[32], tS + 32);
-        tmem_ld_wait();
         const int nvalid = lim - j * kBlockKeys - hf * 64;     // keys of my half the row may see
-        if (__any_sync(0xffffffffu, nvalid < 64)) {            // only the blocks on the diagonal
+        auto load_scores = [&]() {
+          tmem_ld32(&v[0], tS);
+          tmem_ld32(&v[32], tS + 32);
+          tmem_ld_wait();
+          if (__any_sync(0xffffffffu, nvalid < 64)) {          // only the blocks on the diagonal
 #pragma unroll
-          for (int i = 0; i < 64; ++i)
-            if (i >= nvalid) v[i] = -CUDART_INF_F;             // 2^(-inf) = 0 exactly
-        }
-        // The row maximum over both halves, exactly: each thread posts the maximum of its half and
-        // reads its partner's (the scale is positive, so it commutes with max). A row of the last,
+            for (int i = 0; i < 64; ++i)
+              if (i >= nvalid) v[i] = -CUDART_INF_F;           // 2^(-inf) = 0 exactly
+          }
+        };
+        load_scores();
+        // p = 2^(s*scale - m_ref) as bf16, to go over the first 32 columns of my half of S. Any
+        // common reference is exact; p <= 2^threshold keeps the bf16 P and the fp32 sums
+        // comfortable, so the reference only moves (and O is only rescaled) when the block maximum
+        // exceeds it by more than the threshold. The two threads of a row post the maxima of their
+        // halves (the scale is positive, so it commutes with max) and read the same two numbers,
+        // so they take the same decision. After the first block of a unit the exponentials are
+        // taken at once against the reference the row already has, and the maximum rides along
+        // with them: that is nearly always the final answer. P stays in registers until the
+        // decision is known, so the scores are still in TMEM for a warp with a row that does
+        // move: it fetches them again and takes the exponentials once more. A row of the last,
         // diagonal block may be masked completely; it keeps its reference (block 0 always holds
         // key 0, which every row sees).
-        // p = 2^(s*scale - m_ref) as bf16 over the first 32 columns of my half of S (the scores are
-        // in registers). Any common reference is exact; p <= 2^threshold keeps the bf16 P and the
-        // fp32 sums comfortable, so the reference only moves (and O is only rescaled) when the
-        // block maximum exceeds it by more than the threshold. Both threads of a row see the
-        // same numbers and take the same decision. After the first block of a unit the
-        // exponentials are taken at once against the reference the row already has, and the
-        // maximum rides along with them: that is nearly always the final answer, and a warp with
-        // a row that does move simply takes them again.
-        float ls = 0.f, x_max;
+        uint32_t pk[32];
+        float ls, x_max;
         if (j == 0) {
           *xchg_mine = max64(v) * scale;                       // first block of a unit: the maximum itself
+          pair_sync();
+          m_ref = fmaxf(*xchg_mine, *xchg_other);
+          ls = exp_pack(v, scale, -m_ref, pk, x_max);
         } else {
-          ls = exp_store(v, scale, -m_ref, tS, x_max);
+          ls = exp_pack(v, scale, -m_ref, pk, x_max);
           *xchg_mine = x_max + m_ref;                          // largest s*scale of my half
-        }
-        pair_sync();
-        const float m_blk = fmaxf(*xchg_mine, *xchg_other);
-        const bool move = j == 0 || m_blk > m_ref + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, move)) {
-          if (j == 0) {
-            m_ref = m_blk;
-          } else {
+          pair_sync();
+          const float m_blk = fmaxf(*xchg_mine, *xchg_other);
+          const bool move = m_blk > m_ref + kRescaleThreshold;
+          if (__any_sync(0xffffffffu, move)) {
             float alpha = 1.f;
             if (move) {
               alpha = ex2(m_ref - m_blk);
@@ -548,9 +547,12 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
               for (int i = 0; i < 16; ++i) ov[i] *= alpha;
               tmem_st16(tO + c * 16, *reinterpret_cast<const uint32_t(*)[16]>(ov));
             }
+            load_scores();
+            ls = exp_pack(v, scale, -m_ref, pk, x_max);
           }
-          ls = exp_store(v, scale, -m_ref, tS, x_max);
         }
+        tmem_st16(tS, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
+        tmem_st16(tS + 16, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
         l += ls;
         tmem_st_wait();
         tc_fence_before();
