@@ -510,7 +510,8 @@ void fill_device(ts_ctx* c, const ts_step* st, int64_t n_tokens, ts::StepDevice*
   d->scale_log2 = c->scale * 1.4426950408889634f;
   d->append_in_decode = 0;
   d->wait_cycles = c->cfg.wait_limit_cycles > 0 ? (long long)c->cfg.wait_limit_cycles : ts::kWaitCycles;
-  d->append_arrivals = 0;      // set by the mixed launch
+  d->append_ctas = 0;          // both set by the mixed launch
+  d->append_arrivals = 0;
 }
 
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
@@ -609,8 +610,10 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
   }
   // head_dim 128 steps with prefill tiles: the mixed kernel appends the new K/V itself
   const bool append_in_kernel = attention && c->n_prefill_items > 0 && c->cfg.head_dim == 128;
-  // decode-only steps: the unit that reads a row's last page writes the row's new token into it
-  const bool append_in_decode = attention && c->n_prefill_items == 0 && n_items > 0;
+  // decode rows of decode-only steps and of head_dim 128 steps: the unit that reads a row's last
+  // page writes the row's new token into it
+  const bool append_in_decode =
+      attention && n_items > c->n_prefill_items && (c->n_prefill_items == 0 || append_in_kernel);
   d.append_in_decode = append_in_decode;
   if (!append_in_kernel && !append_in_decode) {
     TS_CUDA(c, ts::launch_kv_append(d, stream));
@@ -649,7 +652,11 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
           decode_launched = true;
         }
         if (pe) c->prof_mixed.back() = decode_launched;
-        d.append_arrivals = n_ctas + ((c->cfg.debug_flags & TS_DEBUG_LOSE_APPEND_ARRIVAL) ? 1 : 0);
+        // every CTA appends a share of the prefill rows' tokens (one short round while HBM is still
+        // idle: left to the prefill CTAs alone, the same copies take several times longer next to the
+        // decode streams), but only a CTA about to start on prefill work waits for all of them
+        d.append_ctas = n_ctas;
+        d.append_arrivals = d.append_ctas + ((c->cfg.debug_flags & TS_DEBUG_LOSE_APPEND_ARRIVAL) ? 1 : 0);
         TS_CUDA(c, ts::launch_mixed(d, q_map, c->kv_map, c->kv_tile_map, n_ctas, p, stream));
       } else {
         ts::StepDevice dp = d;

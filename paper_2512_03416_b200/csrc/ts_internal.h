@@ -76,8 +76,9 @@ struct StepDevice {
   int32_t Hq, Hkv, D, n_pages, max_pages_per_req, max_requests;
   float scale_log2;        // softmax scale * log2(e)
   long long wait_cycles;   // limit of every bounded wait of the step's kernels, in clock cycles
-  int32_t append_arrivals; // CTAs the mixed kernel's append barrier waits for: its grid size, or one
-                           // more when ts_config.debug_flags asks for a wait that runs out
+  int32_t append_ctas;     // the first append_ctas CTAs of the mixed kernel append the new tokens of the prefill rows
+  int32_t append_arrivals; // what the mixed kernel's CTAs wait for before their first prefill unit:
+                           // append_ctas, or one more when ts_config.debug_flags asks for a wait that runs out
 };
 
 // Launchers. Each enqueues on `stream` and returns the launch's cudaError_t.
@@ -150,6 +151,7 @@ __device__ __forceinline__ void append_tokens(const StepDevice& s, const int32_t
       const int mid = (lo + hi) >> 1;
       if (row_start[mid] <= tok) lo = mid; else hi = mid;
     }
+    if (s.append_in_decode && row_start[lo + 1] - row_start[lo] == 1) continue;
     const int t = rows[n + lo] + (tok - row_start[lo]);
     const int slot = rows[2 * n + lo];
     const bool index_ok = (unsigned)slot < (unsigned)s.max_requests && (unsigned)(t >> 4) < (unsigned)s.max_pages_per_req;

@@ -32,8 +32,9 @@
 // the epilogue of the current unit.
 // The O rescale is lazy: a row's reference maximum only moves when a block's maximum exceeds it by
 // more than 2^8, so most blocks never touch O.
-// The kernel starts by appending the step's new K/V to the pages itself (every CTA a share of
-// the tokens, then a launch-wide counter barrier), which saves a launch in front of it.
+// The kernel appends the step's new K/V to the pages itself, which saves a launch in front of it:
+// every CTA copies a share of the prefill rows' tokens, and only the CTAs about to start on prefill
+// work wait for all of them; the decode units write their rows' own tokens.
 // Every wait is bounded; a wait that runs out raises TS_DEV_TIMEOUT and the CTA drains.
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -368,6 +369,17 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
     if (tid == 0) {
       misc[1] = 0;
       misc[2] = 0;
+      {   // the prefill rows' new K/V must be in their pages before the first tile is read
+        const volatile int32_t* arrived = s.pf_queue + 2;
+        const long long t0 = clock64();
+        while (*arrived < s.append_arrivals) {
+          if (clock64() - t0 > s.wait_cycles) {
+            atomicOr(s.status, TS_DEV_TIMEOUT);
+            break;
+          }
+        }
+        __threadfence();
+      }
       for (int i = 0; i < BAR_COUNT; ++i) {
         const bool softmax_arrives = (i >= BAR_P_FULL && i < BAR_P_FULL + 2) || (i >= BAR_O_EMPTY && i < BAR_O_EMPTY + 2);
         const bool pair = i >= BAR_PAIR && i < BAR_PAIR + 8;
@@ -401,31 +413,21 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
   };
 
   // ---------------------------------------------------------------- KV append (Sec. 2.1)
-  // Every CTA copies its share of the step's new tokens into their pages, then all CTAs of the
-  // launch meet at a counter (they are all resident: one per SM), so that the attention below
-  // sees every page complete. This replaces a launch of its own in front of the kernel.
+  // The first append_ctas CTAs (all of them, as the host sets it) copy a share of the new tokens of
+  // the prefill rows into their pages and count themselves; a CTA waits for that count only before
+  // its first prefill unit (prefill_setup). The new token of a decode row is written by the decode
+  // unit that reads the row's last page, so the CTAs that stream decode rows go on at once:
+  // nothing they read depends on this append.
   pdl_wait();                  // the previous step's kernels are done with the pool and the counters
-  {
+  if ((int)blockIdx.x < s.append_ctas) {
     int32_t* rows = reinterpret_cast<int32_t*>(smem);   // the window's start is free until the roles begin
     stage_rows(s, rows, tid, kPfThreads);
     cta_sync();
-    append_tokens(s, rows, (int)blockIdx.x * (kPfThreads / 32) + warp, (int)gridDim.x * (kPfThreads / 32), lane);
+    append_tokens(s, rows, (int)blockIdx.x * (kPfThreads / 32) + warp, s.append_ctas * (kPfThreads / 32), lane);
     __threadfence();           // this thread's page writes are visible before the CTA counts itself
     fence_proxy_async();       // and the scratch is handed on to the roles' copies
     cta_sync();
-    if (tid == 0) {
-      atomicAdd(s.pf_queue + 2, 1);
-      const volatile int32_t* arrived = s.pf_queue + 2;
-      const long long t0 = clock64();
-      while (*arrived < s.append_arrivals) {
-        if (clock64() - t0 > s.wait_cycles) {
-          atomicOr(s.status, TS_DEV_TIMEOUT);
-          break;
-        }
-      }
-      __threadfence();
-    }
-    cta_sync();
+    if (tid == 0) atomicAdd(s.pf_queue + 2, 1);
   }
 
   if (warp < kSoftmaxWarps) {
