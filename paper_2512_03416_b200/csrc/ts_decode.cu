@@ -12,8 +12,8 @@ template <int D, int NH, int STAGES>
 __global__ void __launch_bounds__(kDecThreads, 1)
 decode_kernel(const StepDevice s, const __grid_constant__ CUtensorMap kv_map) {
   extern __shared__ unsigned char smem_raw[];
-  const uint32_t base = (dec::smem_u32(smem_raw) + 1023u) & ~1023u;
-  unsigned char* smem = smem_raw + (base - dec::smem_u32(smem_raw));
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* smem = smem_raw + (base - smem_u32(smem_raw));
   pdl_launch_dependents();
   if (threadIdx.x == 0) tma_prefetch_desc(&kv_map);
   pdl_wait();                  // from here on the pool, tables and Q are read

@@ -19,6 +19,7 @@
 
 #include "../../include/tokenscale.h"
 #include "ts_internal.h"
+#include "ts_ptx.h"
 #include "ts_tma.h"
 
 namespace ts {
@@ -30,36 +31,11 @@ constexpr int kDecThreads = kDecWarps * 32;
 
 // Barrier of the kDecThreads decode threads (id 1; id 0 stays with the whole block).
 __device__ __forceinline__ void block_sync() { asm volatile("bar.sync 1, %0;\n" ::"n"(kDecThreads) : "memory"); }
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"(addr));
-}
 __device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {
   uint32_t d;
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(d) : "r"(a));
   return d;
 }
-__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-      "{%0,%1,%2,%3};\n"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
 // Shared-memory image of one page stage (written by TMA with the 128-byte swizzle):
 //   D = 128: [half 0: K 16x128B | V 16x128B][half 1: K | V]   (two copies of 4 KB)
 //   D =  64: [K 16x128B | V 16x128B]                            (one copy of 4 KB)
@@ -256,9 +232,9 @@ __device__ __forceinline__ void decode_units(const StepDevice& s, const CUtensor
       for (int ks = 0; ks < D / 16; ++ks) {
         uint32_t a[4];
         const int mi = lane >> 3;
-        ldsm_x4(a, sp + page_off<D>(0, (mi & 1) * 8 + (lane & 7), 2 * ks + (mi >> 1)));
+        ldmatrix_x4(a, sp + page_off<D>(0, (mi & 1) * 8 + (lane & 7), 2 * ks + (mi >> 1)));
 #pragma unroll
-        for (int nh = 0; nh < NH; ++nh) mma16816((ks & 1) ? sc_odd[nh] : sc[nh], a, qf[nh][ks][0], qf[nh][ks][1]);
+        for (int nh = 0; nh < NH; ++nh) mma_bf16((ks & 1) ? sc_odd[nh] : sc[nh], a, qf[nh][ks][0], qf[nh][ks][1]);
       }
 #pragma unroll
       for (int nh = 0; nh < NH; ++nh) {
@@ -300,17 +276,17 @@ __device__ __forceinline__ void decode_units(const StepDevice& s, const CUtensor
           o[nh][dt][3] *= al1;
         }
         // P^T as the B operand: transpose the two 8x8 (key x head) blocks across the warp
-        pb[nh][0] = movmatrix_t(pack2(s0, s1));
-        pb[nh][1] = movmatrix_t(pack2(s2, s3));
+        pb[nh][0] = movmatrix_t(pack_bf16(s0, s1));
+        pb[nh][1] = movmatrix_t(pack_bf16(s2, s3));
       }
       // ---- O^T += V^T P^T : 16 head_dim rows per m-tile
 #pragma unroll
       for (int dt = 0; dt < D / 16; ++dt) {
         uint32_t a[4];
         const int mi = lane >> 3;
-        ldsm_x4_t(a, sp + page_off<D>(1, (mi >> 1) * 8 + (lane & 7), 2 * dt + (mi & 1)));
+        ldmatrix_x4_trans(a, sp + page_off<D>(1, (mi >> 1) * 8 + (lane & 7), 2 * dt + (mi & 1)));
 #pragma unroll
-        for (int nh = 0; nh < NH; ++nh) mma16816(o[nh][dt], a, pb[nh][0], pb[nh][1]);
+        for (int nh = 0; nh < NH; ++nh) mma_bf16(o[nh][dt], a, pb[nh][0], pb[nh][1]);
       }
       __syncwarp();
       ++n_consumed;

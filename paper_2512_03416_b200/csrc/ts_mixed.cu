@@ -42,6 +42,7 @@
 #include "../../include/tokenscale.h"
 #include "ts_decode_body.h"
 #include "ts_internal.h"
+#include "ts_ptx.h"
 #include "ts_tma.h"
 
 namespace ts {
@@ -98,10 +99,6 @@ constexpr int kSmemBytes = kOffXchg + 2 * 2 * 128 * 4;
 // dynamic window starts on such a boundary; the kernel checks that and refuses to run otherwise
 // (there is no room left for alignment slack).
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory one CTA can opt into");
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
 
 // ---- tcgen05 wrappers
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
@@ -220,10 +217,6 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
 
 // Half a row of a score block: p_i = 2^(x_i), x_i = v_i * scale + neg_m, for the 64 scores in v,
 // as bf16 pairs in pk (the scores are not needed afterwards, so their registers come free as
@@ -241,7 +234,7 @@ __device__ __forceinline__ float exp_pack(const float (&v)[64], float scale, flo
     p0 = ex2(x0);
     p1 = ex2(x1);
     if (i & 1) sum_b = add2(sum_b, pack_f2(p0, p1)); else sum_a = add2(sum_a, pack_f2(p0, p1));
-    pk[i] = pack2(p0, p1);
+    pk[i] = pack_bf16(p0, p1);
   }
   x_max = fmaxf(xm0, xm1);
   float a0, a1;
@@ -584,10 +577,10 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               uint4 wv;
-              wv.x = pack2(ov[8 * i] * inv, ov[8 * i + 1] * inv);
-              wv.y = pack2(ov[8 * i + 2] * inv, ov[8 * i + 3] * inv);
-              wv.z = pack2(ov[8 * i + 4] * inv, ov[8 * i + 5] * inv);
-              wv.w = pack2(ov[8 * i + 6] * inv, ov[8 * i + 7] * inv);
+              wv.x = pack_bf16(ov[8 * i] * inv, ov[8 * i + 1] * inv);
+              wv.y = pack_bf16(ov[8 * i + 2] * inv, ov[8 * i + 3] * inv);
+              wv.z = pack_bf16(ov[8 * i + 4] * inv, ov[8 * i + 5] * inv);
+              wv.w = pack_bf16(ov[8 * i + 6] * inv, ov[8 * i + 7] * inv);
               *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = wv;
             }
           }
@@ -649,8 +642,8 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
         }
         const float inv = 1.f / l;
         uint2 o;
-        o.x = pack2(acc.x * inv, acc.y * inv);
-        o.y = pack2(acc.z * inv, acc.w * inv);
+        o.x = pack_bf16(acc.x * inv, acc.y * inv);
+        o.y = pack_bf16(acc.z * inv, acc.w * inv);
         *reinterpret_cast<uint2*>(s.out + ((size_t)c.token * s.Hq + h) * kD + lane * 4) = o;
       }
     }
