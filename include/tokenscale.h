@@ -423,6 +423,86 @@ int ts_decode_attention_static(int32_t device, int32_t n_q_heads, int32_t n_kv_h
                                const int32_t* kv_len, int32_t n_rows, int32_t n_splits,
                                float softmax_scale, const void* q, void* out, void* cuda_stream);
 
+/*
+ * The decoder layer around the attention step. The paper's velocities are rates of whole model
+ * iterations (prefill velocity, Sec. 3.2: the maximum speed at which input tokens are processed,
+ * bound by GPU compute; Sec. 4.4 profiles the iteration time of a Convertible Decoder against the
+ * TPOT SLO); an iteration runs, for every layer, the projections in front of attention, attention
+ * over the paged KV cache with the append of the new K/V (Sec. 2.1), the output projection and the
+ * MLP. The paper runs Llama-3.1-8B and Qwen-2.5-32B (Sec. 6.1) and describes none of this; the
+ * layer here is the pre-norm block those models share:
+ *      h = rmsnorm(x; w_norm1)            q, k, v = split(h . W_qkv^T); q, k = rope(q, k; position)
+ *      a = ts_mixed_step(q, k, v)         y = x + a . W_o^T
+ *      h2 = rmsnorm(y; w_norm2)           out = y + (silu(h2 . W_gate^T) * (h2 . W_up^T)) . W_down^T
+ * rmsnorm(x; w) = x / sqrt(mean(x^2) + rms_eps) * w per token; rope rotates the pairs (i, i + D/2)
+ * of every query and key head by the angle position * rope_theta^(-2i/D), position = ctx_len + i
+ * for the row's i-th new token; silu(t) = t / (1 + exp(-t)). All tensors are bf16 (the serving
+ * precision, Sec. 6.1): every tensor named above is rounded to bf16 (nearest even) where it is
+ * produced, sums are accumulated in fp32. Weights are [out features][in features], row-major.
+ * head_dim must be 128, hidden a multiple of 64, intermediate a multiple of 128, and the context's
+ * chunk_size > 0 (it sizes the activations).
+ */
+typedef struct ts_layer ts_layer; /* opaque; host memory; used with its ts_ctx, one thread and stream at a time */
+typedef struct {
+  int32_t hidden;           /* model width: columns of x                                        */
+  int32_t intermediate;     /* MLP width                                                        */
+  int32_t max_position;     /* rows of the rotary table: ctx_len + q_len of a row must not exceed it */
+  float rms_eps;            /* 0 => 1e-5                                                        */
+  float rope_theta;         /* 0 => 500000                                                      */
+  const void* w_norm1;      /* DEVICE bf16 [hidden]                                             */
+  const void* w_qkv;        /* DEVICE bf16 [(Hq + 2 Hkv) D][hidden]: query heads, key heads, value heads */
+  const void* w_o;          /* DEVICE bf16 [hidden][Hq D]                                       */
+  const void* w_norm2;      /* DEVICE bf16 [hidden]                                             */
+  const void* w_gate_up;    /* DEVICE bf16 [2 intermediate][hidden] in the order ts_pack_gate_up writes */
+  const void* w_down;       /* DEVICE bf16 [hidden][intermediate]                               */
+  void* workspace;          /* DEVICE, ts_layer_workspace_bytes() bytes, 256-byte aligned, caller-owned: the
+                               rotary table and the layer's activations                         */
+  size_t workspace_bytes;
+} ts_layer_config;          /* all weight pointers 16-byte aligned, caller-owned, only read     */
+
+/* 0 on an unsupported shape. Reads the shape fields of both structs and cfg->chunk_size. */
+size_t ts_layer_workspace_bytes(const ts_config* cfg, const ts_layer_config* layer);
+
+/*
+ * ts_pack_gate_up: writes the gate and up projection weights (DEVICE bf16 [intermediate][hidden]
+ * each) interleaved in blocks of 128 rows -- rows [256 b, 256 b + 128) of the result are gate rows
+ * [128 b, 128 b + 128), the next 128 rows the up rows of the same features -- so that one GEMM
+ * tile holds both halves of a feature and can apply the SiLU gate itself. Asynchronous on
+ * cuda_stream. TS_ERR_INVALID unless intermediate % 128 == 0 and hidden % 8 == 0.
+ */
+int ts_pack_gate_up(const void* w_gate, const void* w_up, void* w_gate_up, int32_t intermediate, int32_t hidden,
+                    void* cuda_stream);
+
+/*
+ * ts_layer_create: binds the weights to a context (the layer's attention runs on the context's
+ * pool and block tables) and enqueues the rotary table's computation on cuda_stream.
+ * TS_ERR_UNSUPPORTED for a shape outside the limits above, TS_ERR_WORKSPACE for a short workspace.
+ * ts_layer_destroy frees host memory only; destroy the layer before its context.
+ */
+int ts_layer_create(ts_ctx* ctx, const ts_layer_config* cfg, void* cuda_stream, ts_layer** out);
+int ts_layer_destroy(ts_layer* layer);
+
+/*
+ * ts_layer_step: one iteration of the layer over the step's rows (slot, q_len, ctx_len as for
+ * ts_mixed_step, which it calls; q, k_new, v_new, out of `step` are ignored). x_in, x_out: DEVICE
+ * bf16 [N][hidden], 16-byte aligned, may not alias. Everything is enqueued on cuda_stream; the
+ * call does not synchronise. Validation is the step's own (nothing is launched on failure), plus
+ * TS_ERR_INVALID when a row reaches past max_position. Updates the context's counters as
+ * ts_mixed_step does.
+ */
+int ts_layer_step(ts_layer* layer, const ts_step* step, const void* x_in, void* x_out, void* cuda_stream);
+int ts_layer_last_cuda_error(const ts_layer* layer);
+
+/*
+ * ts_gemm_bf16: the layer's projection kernel by itself (for measurements and tests):
+ * C[M][N] = (R ? R : 0) + A[M][K] . B[N][K]^T, all DEVICE bf16 row-major and 16-byte aligned, fp32
+ * accumulation, bf16 result. N and K multiples of 8. tile_m: rows of an output tile per thread
+ * block, 128 or 256, 0 = chosen from the shape. device_status: DEVICE int32 the caller has zeroed;
+ * a bounded wait that runs out sets TS_DEV_TIMEOUT there. Asynchronous on cuda_stream.
+ */
+int ts_gemm_bf16(int32_t device, int32_t M, int32_t N, int32_t K, const void* A, const void* B, const void* R,
+                 void* C, int32_t tile_m, int32_t* device_status, void* cuda_stream);
+
 /* The cudaError_t of the most recent failed CUDA call of this context (0 if none). */
 int ts_last_cuda_error(const ts_ctx* ctx);
 

@@ -44,6 +44,14 @@ class ts_config(ctypes.Structure):
                 ("wait_limit_cycles", ctypes.c_int64), ("debug_flags", ctypes.c_int32)]
 
 
+class ts_layer_config(ctypes.Structure):
+    _fields_ = [("hidden", ctypes.c_int32), ("intermediate", ctypes.c_int32), ("max_position", ctypes.c_int32),
+                ("rms_eps", ctypes.c_float), ("rope_theta", ctypes.c_float),
+                ("w_norm1", ctypes.c_void_p), ("w_qkv", ctypes.c_void_p), ("w_o", ctypes.c_void_p),
+                ("w_norm2", ctypes.c_void_p), ("w_gate_up", ctypes.c_void_p), ("w_down", ctypes.c_void_p),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+
+
 class ts_step(ctypes.Structure):
     _fields_ = [("n_rows", ctypes.c_int32), ("flags", ctypes.c_int32),
                 ("slot", _i32p), ("q_len", _i32p), ("ctx_len", _i32p),
@@ -72,7 +80,9 @@ EXPORTS = ["ts_pool_bytes", "ts_workspace_bytes", "ts_create", "ts_destroy", "ts
            "ts_last_device_status", "ts_last_cuda_error", "ts_strerror", "ts_profile_enable",
            "ts_profile_read", "ts_decode_attention_static", "ts_alloc_step", "ts_pick_chunk_size",
            "ts_convertible_prefill_velocity", "ts_reserved_memory", "ts_reserved_pages",
-           "ts_prefiller_instances", "ts_decoder_demand", "ts_regular_decoders", "ts_route_prefill"]
+           "ts_prefiller_instances", "ts_decoder_demand", "ts_regular_decoders", "ts_route_prefill",
+           "ts_layer_workspace_bytes", "ts_pack_gate_up", "ts_layer_create", "ts_layer_destroy", "ts_layer_step",
+           "ts_layer_last_cuda_error", "ts_gemm_bf16"]
 
 _lib = None
 
@@ -139,6 +149,16 @@ def lib() -> ctypes.CDLL:
         L.ts_decode_attention_static.argtypes = [
             ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp,
             ctypes.c_int32, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_float, vp, vp, vp]
+        lcfgp = ctypes.POINTER(ts_layer_config)
+        L.ts_layer_workspace_bytes.restype = ctypes.c_size_t
+        L.ts_layer_workspace_bytes.argtypes = [cfgp, lcfgp]
+        L.ts_pack_gate_up.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, vp]
+        L.ts_layer_create.argtypes = [vp, lcfgp, vp, ctypes.POINTER(vp)]
+        L.ts_layer_destroy.argtypes = [vp]
+        L.ts_layer_step.argtypes = [vp, stepp, vp, vp, vp]
+        L.ts_layer_last_cuda_error.argtypes = [vp]
+        L.ts_gemm_bf16.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp, vp,
+                                   ctypes.c_int32, vp, vp]
         L.ts_strerror.restype = ctypes.c_char_p
         L.ts_strerror.argtypes = [ctypes.c_int]
         for name in EXPORTS:
@@ -355,3 +375,32 @@ def ts_last_cuda_error(ctx) -> int:
 
 def ts_strerror(code: int) -> str:
     return lib().ts_strerror(code).decode()
+
+
+# ------------------------------------------------------------------- the decoder layer around attention
+def ts_layer_workspace_bytes(cfg: ts_config, layer: ts_layer_config) -> int:
+    return lib().ts_layer_workspace_bytes(ctypes.byref(cfg), ctypes.byref(layer))
+
+
+def ts_pack_gate_up(w_gate: int, w_up: int, w_gate_up: int, intermediate: int, hidden: int, stream: int) -> int:
+    return lib().ts_pack_gate_up(w_gate, w_up, w_gate_up, intermediate, hidden, stream)
+
+
+def ts_layer_create(ctx, layer: ts_layer_config, stream: int):
+    """Returns (code, handle)."""
+    h = ctypes.c_void_p()
+    rc = lib().ts_layer_create(ctx, ctypes.byref(layer), stream, ctypes.byref(h))
+    return rc, h
+
+
+def ts_layer_destroy(layer) -> int:
+    return lib().ts_layer_destroy(layer)
+
+
+def ts_layer_step(layer, step: ts_step, x_in: int, x_out: int, stream: int) -> int:
+    return lib().ts_layer_step(layer, ctypes.byref(step), x_in, x_out, stream)
+
+
+def ts_gemm_bf16(device: int, M: int, N: int, K: int, A: int, B: int, R: int, C: int, tile_m: int, status: int,
+                 stream: int) -> int:
+    return lib().ts_gemm_bf16(device, M, N, K, A, B, R or None, C, tile_m, status, stream)

@@ -690,6 +690,21 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
 
 }  // namespace
 
+namespace ts {
+int ctx_view(ts_ctx* c, cudaStream_t stream, CtxView* out) {
+  if (!c || !out) return TS_ERR_INVALID;
+  const int rc = ensure_cuda(c, stream);
+  if (rc != TS_OK) return rc;
+  out->cfg = &c->cfg;
+  out->n_sms = c->n_sms;
+  out->encode_fn = c->encode_fn;
+  out->status = (int32_t*)((char*)c->cfg.workspace + c->L.off_status);
+  out->wait_cycles = c->cfg.wait_limit_cycles > 0 ? (long long)c->cfg.wait_limit_cycles : kWaitCycles;
+  out->max_tokens = c->L.max_tokens;
+  return TS_OK;
+}
+}  // namespace ts
+
 extern "C" {
 
 size_t ts_pool_bytes(const ts_config* cfg) {

@@ -101,6 +101,49 @@ cudaError_t launch_mixed(const StepDevice& s, const CUtensorMap& q_map, const CU
                          const CUtensorMap& kv_tile_map, int n_ctas, int n_prefill_ctas, cudaStream_t stream);
 cudaError_t launch_decode(const StepDevice& s, const CUtensorMap& kv_map, int n_sms, cudaStream_t stream);
 
+// ---- the decoder layer around the attention step: GEMMs and small kernels (ts_gemm.cu, ts_layer_kernels.cu)
+enum { GEMM_EPI_STORE = 0, GEMM_EPI_ROPE = 1, GEMM_EPI_SILU_MUL = 2 };
+// C = A . B^T (+ R), A [M][K], B [N][K] bf16 K-major (their tensor maps travel beside this struct).
+struct GemmArgs {
+  int32_t M, N, K;
+  int32_t epi;              // GEMM_EPI_*
+  uint16_t* C;              // STORE: [M][ldc]; ROPE: the query heads [M][q_cols]; SILU_MUL: [M][ldc], ldc = N / 2
+  const uint16_t* R;        // STORE: residual [M][ldc] added before rounding, or null
+  int32_t ldc;
+  // ROPE (fused QKV projection, head_dim 128): columns [0, q_cols) are query heads -> C, the next
+  // kv_cols key heads -> C2, the last kv_cols value heads -> C3 (not rotated)
+  int32_t q_cols, kv_cols;
+  uint16_t* C2;
+  uint16_t* C3;
+  const int32_t* pos;       // [M] position of every token
+  const float2* rope_table; // [max_position][64] (cos, sin) of pos * theta^(-2i/128)
+  int32_t* status;          // device status word
+  long long wait_cycles;    // limit of every bounded wait
+};
+// What the layer code needs to know of a context (ts_host.cpp fills it in; it also makes sure the
+// context's CUDA set-up has run and its status word is cleared).
+struct CtxView {
+  const ts_config* cfg;
+  int n_sms;
+  void* encode_fn;          // cuTensorMapEncodeTiled
+  int32_t* status;          // device status word of the context
+  long long wait_cycles;
+  int max_tokens;           // most tokens a step may hold
+};
+int ctx_view(ts_ctx* c, cudaStream_t stream, CtxView* out);
+// Tile height (128 or 256 rows per CTA) that finishes an M x N product in the fewest tile-waves.
+int gemm_tile_m(int M, int N, int n_sms);
+cudaError_t launch_gemm(const GemmArgs& g, const CUtensorMap& a_map, const CUtensorMap& b_map, int tile_m, int n_sms,
+                        cudaStream_t stream);
+// out[row] = x[row] / sqrt(mean(x[row]^2) + eps) * gain, bf16 in and out, fp32 inside; width % 8 == 0
+cudaError_t launch_rmsnorm(const uint16_t* x, const uint16_t* gain, uint16_t* out, int rows, int width, float eps,
+                           cudaStream_t stream);
+// table[p][i] = (cos, sin)(p * theta^(-2 i / 128)), p < max_position, i < 64 (computed in fp64)
+cudaError_t launch_rope_table(float2* table, int max_position, float theta, cudaStream_t stream);
+// dst row 256 b + r = gate row 128 b + r, dst row 256 b + 128 + r = up row 128 b + r (r < 128)
+cudaError_t launch_pack_gate_up(const uint16_t* gate, const uint16_t* up, uint16_t* dst, int intermediate, int width,
+                                cudaStream_t stream);
+
 // Programmatic dependent launch: every kernel of a step is launched with the attribute that lets
 // it become resident while its predecessor in the stream is still draining. Each kernel runs its
 // set-up (shared-memory barriers, TMEM allocation, descriptor prefetch), then executes
