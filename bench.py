@@ -42,6 +42,8 @@ WORKLOADS = {
     "config4": (wl.config4, "chunked-prefill continuation, 8B-shaped layer (128 decode rows + 4 chunks of 512 tokens)"),
     "prefill_8192_70b": (None, "one fresh 8192-token prefill chunk alone, 70B-shaped layer (the tile path by itself)"),
     "prefill_2048_8b": (None, "one fresh 2048-token prefill chunk alone, 8B-shaped layer (config3's chunk by itself)"),
+    "layer_8b": (None, "the whole decoder layer (RMSNorm, QKV + rotary, attention, output projection, gated MLP; hidden 4096, "
+                       "intermediate 14336) over config3's batch: 64 decode rows + one fresh 2048-token prefill chunk"),
     "config5": (None, "bursty trace replay, 70B-shaped layer (200 steps, Gamma arrivals CV=4, <=256 decodes, one prefill task at a time)"),
     "config5_chunked": (None, "the same bursty trace under a chunk size of 2304 (2048 prefill tokens + 256 decode rows): "
                               "prompts continue over several steps, up to 4 requests' chunks share a step"),
@@ -242,6 +244,17 @@ def run_reference(args):
     if rank != 0:
         return
     desc = WORKLOADS[args.workload][1]
+    if args.workload == "layer_8b":
+        vals = [layer_cpu_baseline(wl.LLAMA8B, LAYER_8B["hidden"], LAYER_8B["intermediate"]) for _ in range(args.warmup + args.steps)][args.warmup:]
+        value = float(np.mean([v["value"] for v in vals])) if vals else 0.0
+        base = dict(vals[-1], value=value) if vals else None
+        line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": 128.0 / max(value, 1e-9) * 1e3, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": args.workload, "description": desc},
+                "cpu_baseline": base, "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line), flush=True)
+        return
     batch = make_static_batch(args.workload, 0)
     leg = OracleLeg(batch)
     budget = 150.0 / max(1, args.steps + args.warmup)
@@ -428,6 +441,177 @@ def run_static(args, world, rank, local, barrier, workload=None, light=False):
                 extra={"timed_blocks": n_blocks, "timed_region_s": region_s})
 
 
+LAYER_8B = {"hidden": 4096, "intermediate": 14336, "max_position": 16384}
+
+
+def layer_cpu_baseline(s, hidden, inter, n_tokens=128):
+    """The layer oracle (fp64, numpy on all host cores for the projections, the C oracle for the
+    attention) on a bounded sample: one fresh chunk of n_tokens tokens through the whole layer."""
+    import oracle
+    from oracle import layer as OL
+    rng = np.random.default_rng(7)
+    qd, kvd = s.Hq * s.D, s.Hkv * s.D
+
+    def bits(shape, std):
+        return wl.f32_to_bf16_bits((rng.standard_normal(shape, dtype=np.float32) * np.float32(std)))
+
+    wt = dict(w_norm1=bits((hidden,), 1.0), w_qkv=bits((qd + 2 * kvd, hidden), hidden ** -0.5), w_o=bits((hidden, qd), qd ** -0.5),
+              w_norm2=bits((hidden,), 1.0), w_gate=bits((inter, hidden), hidden ** -0.5), w_up=bits((inter, hidden), hidden ** -0.5),
+              w_down=bits((hidden, inter), inter ** -0.5))
+    x = bits((n_tokens, hidden), 1.0)
+    b = wl.make_batch("layer_sample", s, [0], [n_tokens], seed=8, identity_tables=True)
+    pool, tm = b.fresh_pool(), b.table_matrix()
+
+    def attention(q, k, v):
+        return oracle.mixed_step(pool, s.Hq, s.Hkv, s.D, s.P, 1.0 / math.sqrt(s.D), tm, b.ctx_len, b.q_len, q, k, v)
+
+    t0 = time.perf_counter()
+    OL.layer_step(attention, x, wt, OL.positions(b.ctx_len, b.q_len), s.Hq, s.Hkv, s.D)
+    t = time.perf_counter() - t0
+    return {"value": n_tokens / t, "unit": UNIT, "cores": oracle.default_threads(), "kind": "oracle",
+            "sample": f"one fresh chunk of {n_tokens} tokens through the whole layer oracle (fp64), {t:.1f} s"}
+
+
+def run_layer(args, world, rank, local, barrier):
+    """The decoder layer around the attention step (ts_layer_step) on config3's batch, with seeded
+    random weights of the 8B-shaped layer. Timed like run_static; the projection GEMMs are also timed
+    by themselves (ts_gemm_bf16 on the same shapes) for the dominant kernel's roofline."""
+    import torch
+    from paper_2512_03416_b200 import binding as B
+    from paper_2512_03416_b200.harness import LoadedBatch
+    from paper_2512_03416_b200.layer import DecoderLayer
+
+    batch = wl.config3(seed=rank_seed(2, rank))
+    lb = LoadedBatch(batch, device=local, nan_fill=False)
+    s = batch.shape
+    hidden, inter = LAYER_8B["hidden"], LAYER_8B["intermediate"]
+    qd, kvd = s.Hq * s.D, s.Hkv * s.D
+    gen = torch.Generator(device="cuda").manual_seed(rank_seed(71, rank))
+
+    def weight(rows, cols, std):
+        return (torch.randn(rows, cols, generator=gen, device="cuda") * std).to(torch.bfloat16).view(torch.int16)
+
+    def gain():
+        return (1.0 + 0.05 * torch.randn(hidden, generator=gen, device="cuda")).to(torch.bfloat16).view(torch.int16)
+
+    w = dict(w_norm1=gain(), w_qkv=weight(qd + 2 * kvd, hidden, hidden ** -0.5),
+             w_o=weight(hidden, qd, qd ** -0.5), w_norm2=gain(),
+             w_gate=weight(inter, hidden, hidden ** -0.5), w_up=weight(inter, hidden, hidden ** -0.5),
+             w_down=weight(hidden, inter, inter ** -0.5))
+    layer = DecoderLayer(lb.dec, w["w_norm1"], w["w_qkv"], w["w_o"], w["w_norm2"], w["w_gate"], w["w_up"], w["w_down"],
+                         max_position=LAYER_8B["max_position"])
+    del w["w_gate"], w["w_up"]
+    N = batch.n_tokens
+    x_in = (torch.randn(N, hidden, generator=gen, device="cuda")).to(torch.bfloat16).view(torch.int16)
+    x_out = torch.empty_like(x_in)
+    st, _keep = layer.make_step(lb.slots, batch.q_len.tolist(), batch.ctx_len.tolist(), keep_len=True)
+    K, W = args.steps, max(args.warmup, 3)
+    for _ in range(W):
+        layer.step_prepared(st, x_in, x_out)
+    barrier()
+    v0 = lb.dec.velocity()
+    sampler = ClockSampler(local)
+    sampler.start()
+    events = [torch.cuda.Event(enable_timing=True)]
+    barrier()
+    t_host = time.perf_counter()
+    events[0].record()
+    n_blocks = 0
+    while True:
+        for _ in range(K):
+            layer.step_prepared(st, x_in, x_out)
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record()
+        events.append(ev)
+        n_blocks += 1
+        ev.synchronize()
+        if time.perf_counter() - t_host >= MIN_TIMED_S or n_blocks >= MAX_BLOCKS:
+            break
+    barrier()
+    clocks = sampler.stop()
+    block_ms = [events[i].elapsed_time(events[i + 1]) for i in range(n_blocks)]
+    ms_step = reduce_max(float(np.median(block_ms)), world, "cuda") / K
+    region_s = events[0].elapsed_time(events[-1]) * 1e-3
+    attn_launches = int(lb.dec.velocity()["kernel_launches"] - v0["kernel_launches"]) // n_blocks
+    launches = attn_launches + 6 * K                     # two RMSNorm and four GEMM launches per step besides attention's
+    if lb.dec.device_status() != 0:
+        raise SystemExit("the device reported a failure during the timed steps")
+
+    # the four projections by themselves, same shapes, same kernel
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    gemms = {}
+    a_buf = torch.randn(N * max(hidden, inter), generator=gen, device="cuda").to(torch.bfloat16).view(torch.int16)
+    b_buf = (torch.randn(2 * inter * hidden, generator=gen, device="cuda") * hidden ** -0.5).to(torch.bfloat16).view(torch.int16)
+    c_buf = torch.empty(N * 2 * inter, dtype=torch.int16, device="cuda")
+    for name, (n_out, k_in) in {"qkv": (qd + 2 * kvd, hidden), "o": (hidden, qd), "gate_up": (2 * inter, hidden),
+                                "down": (hidden, inter)}.items():
+        tile_m = 128 if name == "qkv" else 0
+        call = lambda: B.ts_gemm_bf16(local, N, n_out, k_in, a_buf.data_ptr(), b_buf.data_ptr(), 0, c_buf.data_ptr(), tile_m,
+                                      status.data_ptr(), stream)
+        for _ in range(3):
+            assert call() == B.TS_OK
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / 20
+        gemms[name] = {"ms": ms, "flops": 2.0 * N * n_out * k_in, "tflops": 2.0 * N * n_out * k_in / ms / 1e9}
+    if int(status.item()) != 0:
+        raise SystemExit("a projection GEMM reported a failure")
+
+    attn_flops, attn_bytes = batch.algorithmic_work()
+    gemm_flops = sum(g["flops"] for g in gemms.values())
+    weight_bytes = 2.0 * ((qd + 2 * kvd) * hidden + hidden * qd + 3 * inter * hidden + 2 * hidden)
+    act_bytes = 2.0 * N * (2 * hidden + 2 * hidden + 2 * (qd + 2 * kvd) + 2 * qd + 2 * hidden + 2 * inter + 2 * hidden)
+    flops, byts = attn_flops + gemm_flops, attn_bytes + weight_bytes + act_bytes
+
+    # end to end: the layer's input starts in pinned host memory and its output returns there
+    hx = x_in.cpu().pin_memory()
+    ho = torch.empty_like(hx).pin_memory()
+    t0 = time.perf_counter()
+    for _ in range(3):
+        x_in.copy_(hx, non_blocking=True); layer.step_prepared(st, x_in, x_out); ho.copy_(x_out, non_blocking=True)
+    torch.cuda.synchronize()
+    est = (time.perf_counter() - t0) / 3
+    Ke = int(min(max(K, math.ceil(MIN_TIMED_S / max(est, 1e-5))), 2000))
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(Ke):
+        x_in.copy_(hx, non_blocking=True)
+        layer.step_prepared(st, x_in, x_out)
+        ho.copy_(x_out, non_blocking=True)
+    torch.cuda.synchronize()
+    e2e_s = reduce_max(time.perf_counter() - t0, world, "cuda")
+    e2e = {"value": aggregate_value(N, world, e2e_s / Ke), "unit": UNIT, "h2d_bytes_per_step": int(hx.numel() * 2),
+           "d2h_bytes_per_step": int(ho.numel() * 2), "steps": Ke, "ms_per_step": e2e_s / Ke * 1e3}
+    layer.close()
+    lb.dec.close()
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = layer_cpu_baseline(s, hidden, inter)
+    peaks, peak_kind = load_peaks()
+    dom = max(gemms.items(), key=lambda kv: kv[1]["ms"])
+    roof = {"bound": "tensor", "achieved": dom[1]["tflops"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+            "frac": dom[1]["tflops"] / peaks["bf16_tflops"], "frac_nominal": dom[1]["tflops"] / 2250.0, "traffic": None,
+            "kernel": f"gemm_kernel ({dom[0]} projection, {N} x {int(dom[1]['flops'] / 2 / N / (hidden if dom[0] != 'down' else inter))} x {hidden if dom[0] != 'down' else inter})",
+            "kernel_ms": dom[1]["ms"], "kernel_ms_source": "events around 20 launches of the kernel alone on the same shape",
+            "peak_source": f"of {peak_kind}",
+            "projections": {k: {"ms": g["ms"], "TFLOPs": g["tflops"], "frac": g["tflops"] / peaks["bf16_tflops"]} for k, g in gemms.items()}}
+    t_hbm, t_tc = byts / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)
+    step_roof = {"t_roof_us": max(t_hbm, t_tc) * 1e6, "t_hbm_us": t_hbm * 1e6, "t_tensor_us": t_tc * 1e6,
+                 "frac": max(t_hbm, t_tc) / (ms_step * 1e-3), "flops": flops, "bytes": byts,
+                 "frac_nominal": max(byts / 8e12, flops / 2.25e15) / (ms_step * 1e-3)}
+    cfg = {"decode_rows": batch.decode_tokens, "prefill_tokens": batch.prefill_tokens, "hidden": hidden, "intermediate": inter,
+           "l2": "weights (435 MB) and the decode rows' K/V (0.77 GB) are larger than L2",
+           "timing": f"median of {n_blocks} blocks of {K} steps, CUDA events around each block, timed region {region_s:.2f} s"}
+    return dict(batch=batch, ms_step=ms_step, tokens=N, prefill_tokens=batch.prefill_tokens, decode_tokens=batch.decode_tokens,
+                launches=launches, clocks=clocks, e2e=e2e, cfg=cfg, steps=K, warmup=W, roofline=roof, step_roofline=step_roof,
+                cpu_baseline=cpu, extra={"timed_blocks": n_blocks, "timed_region_s": region_s})
+
+
 def run_replay(args, world, rank, local, barrier, workload=None, light=False, n_steps=None):
     """config5: the 200-step bursty replay. Every step is issued once, in order (the state evolves);
     warm-up is a full untimed replay on a fresh instance. `light`: no end-to-end leg."""
@@ -566,6 +750,9 @@ def run_ours(args):
     peaks, peak_kind = load_peaks()
 
     def measure(workload, light, n_steps=None):
+        if workload == "layer_8b":
+            r = run_layer(args, world, rank, local, barrier)
+            return r, r["roofline"], r["step_roofline"]
         if workload in REPLAY_TRACE:
             r = run_replay(args, world, rank, local, barrier, workload, light, n_steps)
         else:
@@ -593,7 +780,9 @@ def run_ours(args):
                 if k in ro["extra"]:
                     others[w][k] = ro["extra"][k]
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if args.workload == "layer_8b":
+        cpu_baseline = r.get("cpu_baseline")
+    elif rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = cpu_baseline_leg(r["batch"] if r["batch"] is not None else make_static_batch(args.workload, 0))
     if rank == 0:
         shape = wl.LLAMA70B if args.workload in REPLAY_TRACE or args.workload.endswith("70b") else wl.LLAMA8B
