@@ -6,10 +6,13 @@ TPOT SLO is violated; the largest chunk size before that is used, Eq. 5 turns it
 decoder's prefill Token Velocity and Eq. 6 into the memory to hold back for absorbed prefills.
 This module takes that measurement on ts_mixed_step itself (CUDA events around the step) and
 hands the points to the library's ts_pick_chunk_size / ts_convertible_prefill_velocity /
-ts_reserved_pages. The step is one attention layer: the iteration time used is the measured
-step time times `n_layers`, which understates a full decoder layer (no projections, no MLP).
+ts_reserved_pages. With `layer_dims=(hidden, intermediate)` the measured step is the whole
+decoder layer (ts_layer_step: projections, rotary embedding, attention, MLP, random weights of that
+size) and the iteration time its step time times `n_layers`: a TPOT but for the embedding and the
+output head. Without it the step is the attention layer alone (ts_mixed_step), which understates a
+full layer and so gives an upper bound on the chunk size.
 
-    python -m paper_2512_03416_b200.profiler --shape 8b --decode-rows 64 --layers 32
+    python -m paper_2512_03416_b200.profiler --shape 8b --decode-rows 64 --layers 32 --hidden 4096 --intermediate 14336
 """
 from __future__ import annotations
 
@@ -23,9 +26,29 @@ from . import binding as B
 from . import workloads as wl
 
 
+def _random_layer(lb, shape: wl.Shape, hidden: int, inter: int, max_position: int, seed: int):
+    """A DecoderLayer with seeded random weights of the given size (profiling only needs their shape)."""
+    import torch
+
+    from .layer import DecoderLayer
+
+    gen = torch.Generator(device=lb.device).manual_seed(seed)
+    qd, kvd = shape.Hq * shape.D, shape.Hkv * shape.D
+
+    def w(rows, cols):
+        return (torch.randn(rows, cols, generator=gen, device=lb.device) * cols ** -0.5).to(torch.bfloat16).view(torch.int16)
+
+    def gain():
+        return torch.ones(hidden, device=lb.device).to(torch.bfloat16).view(torch.int16)
+
+    return DecoderLayer(lb.dec, gain(), w(qd + 2 * kvd, hidden), w(hidden, qd), gain(), w(inter, hidden), w(inter, hidden),
+                        w(hidden, inter), max_position=max_position)
+
+
 def measure_step_seconds(shape: wl.Shape, decode_ctx: Sequence[int], prefill_tokens: int, steps: int = 20,
-                         warmup: int = 3, seed: int = 0, device: int = 0) -> float:
-    """Seconds of one ts_mixed_step over the decode rows plus one fresh prefill chunk."""
+                         warmup: int = 3, seed: int = 0, device: int = 0, layer_dims=None) -> float:
+    """Seconds of one step over the decode rows plus one fresh prefill chunk: ts_mixed_step, or
+    ts_layer_step on a layer of `layer_dims = (hidden, intermediate)`."""
     import torch
 
     from .harness import LoadedBatch
@@ -35,32 +58,44 @@ def measure_step_seconds(shape: wl.Shape, decode_ctx: Sequence[int], prefill_tok
     batch = wl.make_batch(f"profile_{prefill_tokens}", shape, ctx, ql, seed + 100,
                           chunk_size=prefill_tokens + len(decode_ctx))
     lb = LoadedBatch(batch, device=device, nan_fill=False)
+    layer = None
     try:
+        step = lb.step_repeatable
+        if layer_dims is not None:
+            hidden, inter = layer_dims
+            layer = _random_layer(lb, shape, hidden, inter, int(ctx.max()) + prefill_tokens + 16, seed + 7)
+            x_in = torch.randn(batch.n_tokens, hidden, device=lb.device).to(torch.bfloat16).view(torch.int16)
+            x_out = torch.empty_like(x_in)
+            st, _keep = layer.make_step(lb.slots, batch.q_len.tolist(), batch.ctx_len.tolist(), keep_len=True)
+            step = lambda: layer.step_prepared(st, x_in, x_out)
         for _ in range(max(warmup, 1)):
-            lb.step_repeatable()
+            step()
         torch.cuda.synchronize(device)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
-            lb.step_repeatable()
+            step()
         e1.record()
         torch.cuda.synchronize(device)
         if lb.dec.device_status() != 0:
             raise RuntimeError("the device reported an error during profiling")
         return e0.elapsed_time(e1) * 1e-3 / steps
     finally:
+        if layer is not None:
+            layer.close()
         lb.dec.close()
 
 
 def profile_chunk_size(shape: wl.Shape, decode_ctx: Sequence[int], candidates: Sequence[int], n_layers: int,
                        tpot_slo_s: float, ttft_slo_s: float, steps: int = 20, seed: int = 0,
-                       device: int = 0) -> Dict:
+                       device: int = 0, layer_dims=None) -> Dict:
     """Grows the prefill chunk over `candidates` (ascending) until the iteration time passes the
     TPOT SLO (Sec. 4.4) and derives Eq. 5 and Eq. 6 from the chunk size found."""
     sizes: List[int] = []
     seconds: List[float] = []
     for t in candidates:
-        sec = measure_step_seconds(shape, decode_ctx, int(t), steps=steps, seed=seed, device=device) * n_layers
+        sec = measure_step_seconds(shape, decode_ctx, int(t), steps=steps, seed=seed, device=device,
+                                   layer_dims=layer_dims) * n_layers
         sizes.append(int(t))
         seconds.append(sec)
         if sec > tpot_slo_s:               # the paper's sweep ends at the first violation
@@ -71,6 +106,7 @@ def profile_chunk_size(shape: wl.Shape, decode_ctx: Sequence[int], candidates: S
         raise ValueError(f"ts_pick_chunk_size: {B.ts_strerror(chunk)}")
     v = B.ts_convertible_prefill_velocity(chunk, float(batch), tpot_slo_s) if chunk > 0 else 0.0
     return {"prefill_tokens": sizes, "iteration_seconds": seconds, "decode_batch_size": batch, "n_layers": n_layers,
+            "step": "ts_layer_step" if layer_dims is not None else "ts_mixed_step",
             "tpot_slo_s": tpot_slo_s, "ttft_slo_s": ttft_slo_s, "chunk_size": chunk,
             "prefill_velocity_tokens_per_s": v,
             "reserved_pages": B.ts_reserved_pages(v, ttft_slo_s, shape.P),
@@ -88,13 +124,16 @@ def main() -> None:
     ap.add_argument("--candidates", type=int, nargs="*",
                     default=[256, 512, 1024, 2048, 3072, 4096, 6144, 8192, 12288, 16384])
     ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--hidden", type=int, default=0, help="with --intermediate: profile the whole layer (ts_layer_step)")
+    ap.add_argument("--intermediate", type=int, default=0)
     args = ap.parse_args()
     shape = wl.LLAMA8B if args.shape == "8b" else wl.LLAMA70B
     rng = np.random.Generator(np.random.Philox(9))
     ctx = np.clip(np.round(args.median_ctx * np.exp(rng.standard_normal(args.decode_rows))), 128,
                   4 * args.median_ctx).astype(np.int32)
     out = profile_chunk_size(shape, ctx, args.candidates, args.layers, args.tpot_ms * 1e-3, args.ttft_ms * 1e-3,
-                             steps=args.steps)
+                             steps=args.steps,
+                             layer_dims=(args.hidden, args.intermediate) if args.hidden and args.intermediate else None)
     print(json.dumps(out))
 
 

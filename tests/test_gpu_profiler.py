@@ -35,3 +35,14 @@ def test_profile_stops_at_the_first_violation():
                                     ttft_slo_s=0.25, steps=3)
     assert r["prefill_tokens"] == [64]                                # the sweep ended at the first point
     assert r["chunk_size"] == 0 and r["prefill_velocity_tokens_per_s"] == 0.0 and r["reserved_pages"] == 0
+
+
+def test_profile_on_the_whole_layer():
+    """The same sweep with ts_layer_step as the measured step: a layer costs more than its attention."""
+    ctx = [300, 500, 64]
+    attn = profiler.profile_chunk_size(wl.LLAMA8B, ctx, [256], n_layers=32, tpot_slo_s=0.1, ttft_slo_s=0.25, steps=5)
+    full = profiler.profile_chunk_size(wl.LLAMA8B, ctx, [256], n_layers=32, tpot_slo_s=0.1, ttft_slo_s=0.25, steps=5,
+                                       layer_dims=(1024, 2048))
+    assert full["step"] == "ts_layer_step" and attn["step"] == "ts_mixed_step"
+    assert full["iteration_seconds"][0] > attn["iteration_seconds"][0] > 0.0
+    assert full["chunk_size"] == velocity.pick_chunk_size(full["prefill_tokens"], full["iteration_seconds"], len(ctx), 0.1)
