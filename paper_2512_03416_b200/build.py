@@ -8,7 +8,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libtokenscale.so")
 SOURCES = ["ts_host.cpp", "ts_layer.cpp", "ts_kernels.cu", "ts_decode.cu", "ts_mixed.cu", "ts_gemm.cu", "ts_layer_kernels.cu"]
-HEADERS = [os.path.join(CSRC, "ts_internal.h"), os.path.join(CSRC, "ts_tma.h"), os.path.join(CSRC, "ts_ptx.h"), os.path.join(CSRC, "ts_decode_body.h"),
+HEADERS = [os.path.join(CSRC, "ts_internal.h"), os.path.join(CSRC, "ts_tma.h"), os.path.join(CSRC, "ts_ptx.h"), os.path.join(CSRC, "ts_tc.h"), os.path.join(CSRC, "ts_decode_body.h"),
            os.path.join(PKG_DIR, "..", "include", "tokenscale.h")]
 
 

@@ -23,6 +23,7 @@
 #include "../../include/tokenscale.h"
 #include "ts_internal.h"
 #include "ts_ptx.h"
+#include "ts_tc.h"
 #include "ts_tma.h"
 
 namespace ts {
@@ -33,65 +34,11 @@ constexpr int kBN = 256, kBK = 64;
 constexpr int kABytes = 128 * kBK * 2;          // one 128-row operand block: 16 KB
 constexpr int kBBytes = kBN * kBK * 2;          // the 256-row weight block: 32 KB
 
-__device__ __forceinline__ void tmem_alloc512(uint32_t smem_dst) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;\n" ::"r"(smem_dst) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc512(uint32_t taddr) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;\n" ::"r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
-__device__ __forceinline__ uint32_t elect_one() {
-  uint32_t pred;
-  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(pred));
-  return pred;
-}
-__device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t issue) {
-  asm volatile(
-      "{\n.reg .pred q;\nsetp.ne.u32 q, %1, 0;\n"
-      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n" ::"r"(bar),
-      "r"(issue)
-      : "memory");
-}
-__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate,
-                                       uint32_t issue) {
-  asm volatile(
-      "{\n.reg .pred p, q;\nsetp.ne.u32 p, %4, 0;\nsetp.ne.u32 q, %5, 0;\n"
-      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d),
-      "l"(a), "l"(b), "r"(idesc), "r"(accumulate), "r"(issue)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(float* v, uint32_t taddr) {
-  uint32_t* r = reinterpret_cast<uint32_t*>(v);
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,"
-      "%27,%28,%29,%30,%31}, [%32];\n"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
-        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
-        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
-        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n" ::"r"(dst),
       "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
       : "memory");
-}
-// Shared-memory matrix descriptor of a K-major operand block, 128-byte swizzle, 1024 bytes between
-// groups of eight rows.
-__device__ __forceinline__ uint64_t smem_desc_k(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr >> 4) & 0x3FFF);
-  d |= (uint64_t)((1024 >> 4) & 0x3FFF) << 32;
-  d |= (uint64_t)1 << 46;   // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;   // 128-byte swizzle
-  return d;
 }
 // bf16 x bf16 -> fp32, M = 128, N = 256, both operands K-major
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
@@ -136,7 +83,7 @@ gemm_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap a_map, const _
     mbar_init(bar(BAR_ACC_EMPTY + 1), 128);
     mbar_init_fence();
   }
-  if (warp == 1) tmem_alloc512(base + kOffBar + (2 * kStages + 4) * 8);
+  if (warp == 1) tmem_alloc(base + kOffBar + (2 * kStages + 4) * 8, 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -200,10 +147,10 @@ gemm_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap a_map, const _
         iwait(BAR_FULL + st, (it / kStages) & 1);
         tc_fence_after();
         if (!dead) {
-          const uint64_t b_desc = smem_desc_k(base + st * kStageBytes + kMB * kABytes);
+          const uint64_t b_desc = smem_desc(base + st * kStageBytes + kMB * kABytes, 0, 1024);
 #pragma unroll
           for (int mb = 0; mb < kMB; ++mb) {
-            const uint64_t a_desc = smem_desc_k(base + st * kStageBytes + mb * kABytes);
+            const uint64_t a_desc = smem_desc(base + st * kStageBytes + mb * kABytes, 0, 1024);
 #pragma unroll
             for (int ks = 0; ks < kBK / 16; ++ks)          // 16 of K = 32 bytes along the swizzled row
               mma_ss(tmem + (kMB == 1 ? buf : mb) * 256, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), kIdesc,
@@ -331,7 +278,7 @@ gemm_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap a_map, const _
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc512(tmem);
+  if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
 template <int TILE_M, int EPI>
