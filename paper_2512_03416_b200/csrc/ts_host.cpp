@@ -527,12 +527,15 @@ bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 //           middle is taken (its ends are the sensitive ones).
 //   G >  4: measured fraction of the full-chip rate by SM count, linear in between:
 //           48 0.475, 64 0.62, 74 0.715, 84 0.78, 100 0.85, 116 0.92, 132 0.95, 148 1
+// A prefill CTA starts on its first unit once the prefill rows' new tokens are in their pages,
+// which next to the decode streams takes ~8 us plus ~11 ns per token.
 int choose_prefill_ctas(const ts_ctx* c, int n_ctas, double prefill_block_pairs, double prefill_units,
-                        double decode_bytes, double decode_units) {
+                        double decode_bytes, double decode_units, double prefill_tokens) {
   static const double kSm8[] = {0, 48, 64, 74, 84, 100, 116, 132, 148};
   static const double kRate8[] = {0, 0.475, 0.62, 0.715, 0.78, 0.85, 0.92, 0.95, 1.0};
   const bool wide = c->G > 4;
   const double w_pf = prefill_block_pairs * 2.1 + prefill_units * 2.0;
+  const double t_append = 8.0 + 0.011 * prefill_tokens;
   const double t_dec_full = decode_bytes / 6.1e6;   // us at 6.1 TB/s
   const double unit_bytes = decode_bytes / std::max(1.0, decode_units);
   const double sm_rate = unit_bytes / (unit_bytes / 70e3 + 2.0);   // bytes per us and SM
@@ -548,7 +551,7 @@ int choose_prefill_ctas(const ts_ctx* c, int n_ctas, double prefill_block_pairs,
     } else {
       td = std::max(t_dec_full, decode_bytes / ((double)(n_ctas - p) * sm_rate));
     }
-    return std::max(td, (w_pf + (double)(n_ctas - p) * td) / n_ctas);
+    return std::max(td, (w_pf + (double)p * t_append + (double)(n_ctas - p) * td) / n_ctas);
   };
   int best = 0;
   double best_t = 1e30;
@@ -644,7 +647,8 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
             for (int i = c->n_prefill_items; i < n_items; ++i)
               bytes += (double)(c->items[i].k_end - c->items[i].k_begin);
             bytes *= 2.0 * c->cfg.n_kv_heads * c->cfg.head_dim * 2.0;
-            p = choose_prefill_ctas(c, n_ctas, pairs * c->cfg.n_kv_heads, (double)pf_units, bytes, (double)dec_units);
+            p = choose_prefill_ctas(c, n_ctas, pairs * c->cfg.n_kv_heads, (double)pf_units, bytes, (double)dec_units,
+                                    (double)n_prefill);
           }
           p = (int)std::min<long long>(p, pf_units);
           p = std::min(p, n_ctas - 1);                         // at least one CTA runs the decode splits
@@ -652,9 +656,9 @@ int run_step(ts_ctx* c, const ts_step* st, void* cuda_stream, bool attention) {
           decode_launched = true;
         }
         if (pe) c->prof_mixed.back() = decode_launched;
-        // every CTA appends a share of the prefill rows' tokens (one short round while HBM is still
-        // idle: left to the prefill CTAs alone, the same copies take several times longer next to the
-        // decode streams), but only a CTA about to start on prefill work waits for all of them
+        // every CTA appends a share of the prefill rows' tokens (in a CTA that streams decode rows
+        // first its loader warpgroup does, so the page stream starts with the kernel), but only a
+        // CTA about to start on prefill work waits for all of them
         d.append_ctas = n_ctas;
         d.append_arrivals = d.append_ctas + ((c->cfg.debug_flags & TS_DEBUG_LOSE_APPEND_ARRIVAL) ? 1 : 0);
         TS_CUDA(c, ts::launch_mixed(d, q_map, c->kv_map, c->kv_tile_map, n_ctas, p, stream));

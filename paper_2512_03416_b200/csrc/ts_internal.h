@@ -76,7 +76,7 @@ struct StepDevice {
   int32_t Hq, Hkv, D, n_pages, max_pages_per_req, max_requests;
   float scale_log2;        // softmax scale * log2(e)
   long long wait_cycles;   // limit of every bounded wait of the step's kernels, in clock cycles
-  int32_t append_ctas;     // the first append_ctas CTAs of the mixed kernel append the new tokens of the prefill rows
+  int32_t append_ctas;     // CTAs of the mixed kernel that append the new tokens of the prefill rows: all of them
   int32_t append_arrivals; // what the mixed kernel's CTAs wait for before their first prefill unit:
                            // append_ctas, or one more when ts_config.debug_flags asks for a wait that runs out
 };
@@ -182,12 +182,52 @@ __device__ __forceinline__ void stage_rows(const StepDevice& s, int32_t* rows, i
   }
 }
 __host__ __device__ inline size_t staged_rows_bytes(int n_rows) { return (size_t)3 * (n_rows + 1) * sizeof(int32_t); }
+// One token: its K and V for all KV heads go to position t of the request in table row `slot`.
+__device__ __forceinline__ void append_one(const StepDevice& s, int tok, int t, int slot, int lane) {
+  const int cpr = s.D / 8;                      // chunks per (token, head) row
+  const int per_tok = 2 * s.Hkv * cpr;
+  const bool index_ok = (unsigned)slot < (unsigned)s.max_requests && (unsigned)(t >> 4) < (unsigned)s.max_pages_per_req;
+  int page = -1;
+  for (int base = 0; base < per_tok; base += 256) {
+    uint4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int c = base + u * 32 + lane;
+      if (c < per_tok) {
+        const int kv = c / (s.Hkv * cpr);
+        const int rem = c - kv * s.Hkv * cpr;
+        const int head = rem / cpr, ch = rem % cpr;
+        v[u] = *reinterpret_cast<const uint4*>((kv ? s.v_new : s.k_new) + ((size_t)tok * s.Hkv + head) * s.D + ch * 8);
+      }
+    }
+    if (base == 0) {
+      if (!index_ok) {
+        if (lane == 0) atomicOr(s.status, TS_DEV_BAD_INDEX);
+        break;
+      }
+      page = s.table[(size_t)slot * s.max_pages_per_req + (t >> 4)];
+      if ((unsigned)page >= (unsigned)s.n_pages) {
+        if (lane == 0) atomicOr(s.status, TS_DEV_BAD_PAGE);
+        break;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int c = base + u * 32 + lane;
+      if (c < per_tok) {
+        const int kv = c / (s.Hkv * cpr);
+        const int rem = c - kv * s.Hkv * cpr;
+        const int head = rem / cpr, ch = rem % cpr;
+        uint16_t* dst = s.pool + ((((size_t)page * 2 + kv) * s.Hkv + head) * kPageSize + (t & 15)) * s.D + ch * 8;
+        *reinterpret_cast<uint4*>(dst) = v[u];
+      }
+    }
+  }
+}
 __device__ __forceinline__ void append_tokens(const StepDevice& s, const int32_t* rows, int first_warp, int n_warps,
                                               int lane) {
   const int n = s.n_rows + 1;
   const int32_t* row_start = rows;
-  const int cpr = s.D / 8;                      // chunks per (token, head) row
-  const int per_tok = 2 * s.Hkv * cpr;
   for (int tok = first_warp; tok < s.n_tokens; tok += n_warps) {
     int lo = 0, hi = s.n_rows;                  // row of this token: last r with row_start[r] <= tok
     while (hi - lo > 1) {
@@ -195,45 +235,20 @@ __device__ __forceinline__ void append_tokens(const StepDevice& s, const int32_t
       if (row_start[mid] <= tok) lo = mid; else hi = mid;
     }
     if (s.append_in_decode && row_start[lo + 1] - row_start[lo] == 1) continue;
-    const int t = rows[n + lo] + (tok - row_start[lo]);
-    const int slot = rows[2 * n + lo];
-    const bool index_ok = (unsigned)slot < (unsigned)s.max_requests && (unsigned)(t >> 4) < (unsigned)s.max_pages_per_req;
-    int page = -1;
-    for (int base = 0; base < per_tok; base += 256) {
-      uint4 v[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int c = base + u * 32 + lane;
-        if (c < per_tok) {
-          const int kv = c / (s.Hkv * cpr);
-          const int rem = c - kv * s.Hkv * cpr;
-          const int head = rem / cpr, ch = rem % cpr;
-          v[u] = *reinterpret_cast<const uint4*>((kv ? s.v_new : s.k_new) + ((size_t)tok * s.Hkv + head) * s.D + ch * 8);
-        }
-      }
-      if (base == 0) {
-        if (!index_ok) {
-          if (lane == 0) atomicOr(s.status, TS_DEV_BAD_INDEX);
-          break;
-        }
-        page = s.table[(size_t)slot * s.max_pages_per_req + (t >> 4)];
-        if ((unsigned)page >= (unsigned)s.n_pages) {
-          if (lane == 0) atomicOr(s.status, TS_DEV_BAD_PAGE);
-          break;
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int c = base + u * 32 + lane;
-        if (c < per_tok) {
-          const int kv = c / (s.Hkv * cpr);
-          const int rem = c - kv * s.Hkv * cpr;
-          const int head = rem / cpr, ch = rem % cpr;
-          uint16_t* dst = s.pool + ((((size_t)page * 2 + kv) * s.Hkv + head) * kPageSize + (t & 15)) * s.D + ch * 8;
-          *reinterpret_cast<uint4*>(dst) = v[u];
-        }
-      }
-    }
+    append_one(s, tok, rows[n + lo] + (tok - row_start[lo]), rows[2 * n + lo], lane);
+  }
+}
+// The same for the tokens of the prefill work items only (they cover every token of every row with
+// more than one new token exactly once, `tokens_per_item` at most each): nothing to stage and no
+// search, the item names the row and the position. Warps `first_warp`, `first_warp + n_warps`, ...
+__device__ __forceinline__ void append_prefill_items(const StepDevice& s, int tokens_per_item, int first_warp, int n_warps,
+                                                     int lane) {
+  const int total = s.n_prefill_items * tokens_per_item;
+  for (int w = first_warp; w < total; w += n_warps) {
+    const WorkItem it = s.items[w / tokens_per_item];
+    const int j = w % tokens_per_item;
+    if (j >= it.q_count) continue;
+    append_one(s, s.row_tok0[it.row] + it.q_begin + j, it.k_end - it.q_count + j, s.row_slot[it.row], lane);
   }
 }
 // Log-sum-exp merge of the splits of one (token, head) for head_dim element d: the exact merge

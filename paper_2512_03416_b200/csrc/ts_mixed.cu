@@ -33,8 +33,9 @@
 // The O rescale is lazy: a row's reference maximum only moves when a block's maximum exceeds it by
 // more than 2^8, so most blocks never touch O.
 // The kernel appends the step's new K/V to the pages itself, which saves a launch in front of it:
-// every CTA copies a share of the prefill rows' tokens, and only the CTAs about to start on prefill
-// work wait for all of them; the decode units write their rows' own tokens.
+// every CTA copies a share of the prefill rows' tokens (in a CTA that streams decode rows first, the
+// loader warpgroup does, next to the stream), and only the CTAs about to start on prefill work wait
+// for all of them; the decode units write their rows' own tokens.
 // Every wait is bounded; a wait that runs out raises TS_DEV_TIMEOUT and the CTA drains.
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -303,28 +304,36 @@ mixed_kernel(const StepDevice s, const __grid_constant__ CUtensorMap q_map,
     cta_sync();
     tc_fence_after();
   };
+  // ---------------------------------------------------------------- KV append (Sec. 2.1)
+  // Every CTA copies a share of the new tokens of the prefill rows into their pages, straight from
+  // the prefill work items (which cover those tokens exactly once), and counts itself; a CTA waits
+  // for that count only before its first prefill unit (prefill_setup). In a CTA that takes prefill
+  // units from the start all twenty warps copy. In a CTA that streams decode rows first only the
+  // fifth warpgroup copies (aux_setup) while warps 0-7 are already on their decode units: nothing
+  // those read depends on this append (the new token of a decode row is written by the decode unit
+  // that reads the row's last page), so the page stream starts with the kernel.
+  constexpr int kWarpsAll = kPfThreads / 32, kWarpsAux = 4;
+  const int append_warps = n_prefill_ctas * kWarpsAll + ((int)gridDim.x - n_prefill_ctas) * kWarpsAux;
   // The fifth warpgroup (loaders, MMA issuer, Q loader): gives registers to the softmax warpgroups
-  // and, in a decode-first CTA, waits while warps 0-7 run the CTA's decode units.
+  // and, in a decode-first CTA, appends and then waits while warps 0-7 run the CTA's decode units.
   auto aux_setup = [&]() {
     reg_dec<kRegsAux>();
-    if (decode_first) cta_sync();
+    if (decode_first) {
+      append_prefill_items(s, 2 * tile_tokens,
+                           n_prefill_ctas * kWarpsAll + ((int)blockIdx.x - n_prefill_ctas) * kWarpsAux + (warp - kSoftmaxWarps),
+                           append_warps, lane);
+      __threadfence();         // this thread's page writes are visible before the CTA counts itself
+      asm volatile("bar.sync 2, 128;\n" ::: "memory");
+      if (tid == kSoftmaxWarps * 32) atomicAdd(s.pf_queue + 2, 1);
+      cta_sync();
+    }
     prefill_setup();
   };
 
-  // ---------------------------------------------------------------- KV append (Sec. 2.1)
-  // The first append_ctas CTAs (all of them, as the host sets it) copy a share of the new tokens of
-  // the prefill rows into their pages and count themselves; a CTA waits for that count only before
-  // its first prefill unit (prefill_setup). The new token of a decode row is written by the decode
-  // unit that reads the row's last page, so the CTAs that stream decode rows go on at once:
-  // nothing they read depends on this append.
   pdl_wait();                  // the previous step's kernels are done with the pool and the counters
-  if ((int)blockIdx.x < s.append_ctas) {
-    int32_t* rows = reinterpret_cast<int32_t*>(smem);   // the window's start is free until the roles begin
-    stage_rows(s, rows, tid, kPfThreads);
-    cta_sync();
-    append_tokens(s, rows, (int)blockIdx.x * (kPfThreads / 32) + warp, s.append_ctas * (kPfThreads / 32), lane);
-    __threadfence();           // this thread's page writes are visible before the CTA counts itself
-    fence_proxy_async();       // and the scratch is handed on to the roles' copies
+  if (!decode_first) {
+    append_prefill_items(s, 2 * tile_tokens, (int)blockIdx.x * kWarpsAll + warp, append_warps, lane);
+    __threadfence();
     cta_sync();
     if (tid == 0) atomicAdd(s.pf_queue + 2, 1);
   }
