@@ -34,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the workload's dominant kernel, from
 # the ncu captures summarised under profiles/ (decode_kernel on config2, mixed_kernel on config3).
 # An entry is dropped (null in the output) when its kernel has changed since the capture.
-KERNEL_TRAFFIC_BYTES = {"config2": 7.746e8, "config3": 8.406e8, "prefill_8192_70b": 2.859e8}
+KERNEL_TRAFFIC_BYTES = {"config2": 7.746e8, "config3": 8.415e8, "prefill_8192_70b": 2.873e8}
 
 WORKLOADS = {
     "config2": (wl.config2, "decode-only batch, 8B-shaped layer (64 decode rows, ctx lognormal median 2048)"),
